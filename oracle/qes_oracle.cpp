@@ -1,0 +1,387 @@
+// QES parameter-pass oracle.  TEST INFRASTRUCTURE ONLY.
+//
+// A plain, slow, scalar CPU statement of what the Quantized Evolution Strategies
+// parameter pass computes, written from the paper (Eq. 3 stochastic rounding,
+// Eq. 4 boundary gate, Eq. 5 discrete gradient, Eqs. 6-8 error feedback,
+// Algorithm 1 stored residual, Algorithm 2 stateless seed replay).  Only tests,
+// the smoke check and the CPU-baseline leg of the benchmark may call it.  It
+// shares no code, header, table or constant generator with the CUDA library.
+//
+// The paper says only "RNG(seed)"; the generator contract implemented here is
+//   Philox4x32-10 (Salmon et al., "Parallel random numbers: as easy as 1, 2, 3")
+//   key = (lo32(seed), hi32(seed)), counter = (lo32(p), hi32(p), 0, 0), p = J >> 1
+//   where J is the global element index; one call serves elements 2p and 2p+1.
+//   words r0,r1 -> Box-Muller pair, words r2,r3 -> the two Bernoulli uniforms.
+// Two tiers:
+//   tier 0 ("plain"): Gaussian in double with libm log/sqrt/sin/cos.
+//   tier 1 ("spec") : Gaussian by a fixed sequence of IEEE fp32 operations
+//                     ("BM24") that a GPU can reproduce bit for bit.
+// Everything after the noise sample (sum, u, round, gate, residual) is double.
+//
+// Build: g++ -O2 -std=c++17 -ffp-contract=off -fPIC -shared -pthread
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <thread>
+#include <vector>
+#include <algorithm>
+
+namespace {
+
+// ---------------------------------------------------------------- Philox4x32-10
+struct U4 { uint32_t v[4]; };
+
+U4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0, uint32_t k1) {
+    const uint64_t M0 = 0xD2511F53ull, M1 = 0xCD9E8D57ull;
+    for (int round = 0; round < 10; ++round) {
+        uint64_t p0 = M0 * (uint64_t)c0;
+        uint64_t p1 = M1 * (uint64_t)c2;
+        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        uint32_t n1 = (uint32_t)p1;
+        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        uint32_t n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        k0 += 0x9E3779B9u;   // golden-ratio Weyl step
+        k1 += 0xBB67AE85u;   // sqrt(3)-1 Weyl step
+    }
+    return U4{{c0, c1, c2, c3}};
+}
+
+inline uint32_t f2u(float f) { uint32_t u; std::memcpy(&u, &f, 4); return u; }
+inline float u2f(uint32_t u) { float f; std::memcpy(&f, &u, 4); return f; }
+
+// ---------------------------------------------------------------- BM24 (tier 1)
+// Radius R = sqrt(-2 ln u1), u1 = n / 2^24, n = (r0 >> 8) + 1 in [1, 2^24].
+float bm24_radius(uint32_t r0) {
+    uint32_t n = (r0 >> 8) + 1u;
+    float nf = (float)n;                       // exact: n <= 2^24
+    uint32_t ib = f2u(nf);
+    uint32_t a = ib - 0x3f3504f3u;             // bits of sqrt(1/2)
+    uint32_t e = a >> 23;                      // 0..24
+    float m = u2f(ib - (e << 23));             // [sqrt(1/2), sqrt(2))
+    float f = m - 1.0f;                        // exact
+    // P(f) ~ -2 log1p(f) / f, degree 8, Horner with fused multiply-add
+    float P = -0x1.6eff90p-3f;
+    P = std::fmaf(P, f,  0x1.289862p-2f);
+    P = std::fmaf(P, f, -0x1.318204p-2f);
+    P = std::fmaf(P, f,  0x1.52d0d4p-2f);
+    P = std::fmaf(P, f, -0x1.98bf96p-2f);
+    P = std::fmaf(P, f,  0x1.0007bap-1f);
+    P = std::fmaf(P, f, -0x1.555780p-1f);
+    P = std::fmaf(P, f,  0x1.fffff2p-1f);
+    P = std::fmaf(P, f, -0x1.000000p+1f);
+    float p = f * P;                           // -2 ln m
+    float ef = (float)(int)(24u - e);
+    float t = std::fmaf(ef, 0x1.62e430p+0f, p); // + (24-e) * 2 ln 2
+    return std::sqrt(t);                       // correctly rounded fp32 sqrt
+}
+
+// (cos, sin) of theta = 2 pi u2, u2 = k / 2^24, k = r1 >> 8.
+void bm24_cossin(uint32_t r1, float* c_out, float* s_out) {
+    uint32_t k = r1 >> 8;
+    uint32_t q = (k + 0x200000u) >> 22;        // nearest quarter turn, 0..4
+    int32_t j = (int32_t)k - (int32_t)(q << 22); // [-2^21, 2^21)
+    float y = (float)j * 0x1p-22f;             // exact; angle = (pi/2) y, |y| <= 1/2
+    float z = y * y;
+    float sp = -0x1.2d9bb8p-8f;
+    sp = std::fmaf(sp, z,  0x1.465ec6p-4f);
+    sp = std::fmaf(sp, z, -0x1.4abbbap-1f);
+    sp = std::fmaf(sp, z,  0x1.921fb6p+0f);
+    float sn = y * sp;
+    float cs = -0x1.4e5ed6p-6f;
+    cs = std::fmaf(cs, z,  0x1.03af5cp-2f);
+    cs = std::fmaf(cs, z, -0x1.3bd392p+0f);
+    cs = std::fmaf(cs, z,  1.0f);
+    switch (q & 3u) {
+        case 0: *c_out =  cs; *s_out =  sn; break;
+        case 1: *c_out = -sn; *s_out =  cs; break;
+        case 2: *c_out = -cs; *s_out = -sn; break;
+        default:*c_out =  sn; *s_out = -cs; break;
+    }
+}
+
+// Eq. 3 in fp32: delta = floor(x) + [v < x - floor(x)], then the 4-bit range of
+// the perturbation tensor (App. A "4-bit stochastically rounded perturbation").
+int stochastic_round_f32(float x, uint32_t rword) {
+    float fl = std::floor(x);
+    float frac = x - fl;
+    float v = (float)(rword >> 8) * 0x1p-24f;  // exact, [0,1)
+    int d = (int)fl + (v < frac ? 1 : 0);
+    return std::min(7, std::max(-8, d));
+}
+
+struct PairNoise { int delta[2]; double x[2]; bool near[2]; };
+
+const double kPi = 3.14159265358979323846;
+
+// Both discrete perturbations of pair p for one seed.  sig[] = sigma_eff of the
+// even and odd element.  tier 0 also flags samples whose decision lies within
+// tau of a floor boundary or of the Bernoulli threshold.
+PairNoise pair_noise(uint64_t seed, uint64_t p, const float sig[2], int tier, double tau) {
+    U4 r = philox4x32_10((uint32_t)p, (uint32_t)(p >> 32), 0u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32));
+    PairNoise out;
+    if (tier == 1) {
+        float R = bm24_radius(r.v[0]);
+        float cs, sn;
+        bm24_cossin(r.v[1], &cs, &sn);
+        float trig[2] = {cs, sn};
+        for (int h = 0; h < 2; ++h) {
+            float rho = sig[h] * R;
+            float x = rho * trig[h];
+            out.delta[h] = stochastic_round_f32(x, r.v[2 + h]);
+            out.x[h] = (double)x;
+            out.near[h] = false;
+        }
+    } else {
+        double u1 = (double)((r.v[0] >> 8) + 1u) / 16777216.0;
+        double u2 = (double)(r.v[1] >> 8) / 16777216.0;
+        double R = std::sqrt(-2.0 * std::log(u1));
+        double th = 2.0 * kPi * u2;
+        double trig[2] = {std::cos(th), std::sin(th)};
+        for (int h = 0; h < 2; ++h) {
+            double x = (double)sig[h] * R * trig[h];
+            double fl = std::floor(x);
+            double frac = x - fl;
+            double v = (double)(r.v[2 + h] >> 8) / 16777216.0;
+            int d = (int)fl + (v < frac ? 1 : 0);
+            out.delta[h] = std::min(7, std::max(-8, d));
+            out.x[h] = x;
+            out.near[h] = (frac < tau) || (frac > 1.0 - tau) || (std::fabs(frac - v) < tau);
+        }
+    }
+    return out;
+}
+
+// ---------------------------------------------------------------- storage
+// IEEE binary16 -> float, written out (no hardware half type).
+float half_to_float(uint16_t h) {
+    uint32_t sign = (uint32_t)(h >> 15) << 31;
+    int exp = (h >> 10) & 0x1f;
+    uint32_t man = h & 0x3ffu;
+    if (exp == 0) {
+        if (man == 0) return u2f(sign);
+        float v = std::ldexp((float)man, -24);       // subnormal: man * 2^-24
+        return (h >> 15) ? -v : v;
+    }
+    if (exp == 31) return u2f(sign | 0x7f800000u | (man << 13));
+    return u2f(sign | ((uint32_t)(exp + 112) << 23) | (man << 13));
+}
+
+// Row-major [rows, cols].  INT4: two codes per byte, even column in the low
+// nibble, two's complement.  INT8: one signed byte per code.
+int load_code(const uint8_t* packed, int bits, int64_t j) {
+    if (bits == 8) return (int)(int8_t)packed[j];
+    uint8_t byte = packed[j >> 1];
+    int nib = (j & 1) ? (byte >> 4) : (byte & 0xf);
+    return nib >= 8 ? nib - 16 : nib;
+}
+void store_code(uint8_t* packed, int bits, int64_t j, int code) {
+    if (bits == 8) { packed[j] = (uint8_t)(int8_t)code; return; }
+    uint8_t nib = (uint8_t)(code & 0xf);
+    uint8_t& b = packed[j >> 1];
+    b = (j & 1) ? (uint8_t)((b & 0x0f) | (nib << 4)) : (uint8_t)((b & 0xf0) | nib);
+}
+
+struct Tensor { int32_t bits, qmin, qmax, group_size; int64_t rows, cols; uint64_t elem_offset; };
+struct HParams { float sigma, lr, gamma; int32_t n_pop, sigma_unit, boundary_mode; };
+
+float sigma_eff(const Tensor& t, const HParams& hp, const uint16_t* scales, int64_t j) {
+    if (hp.sigma_unit == 0) return hp.sigma;                    // sigma in grid steps
+    int64_t row = j / t.cols, col = j % t.cols;
+    int64_t g = (t.group_size > 0) ? row * (t.cols / t.group_size) + col / t.group_size : row;
+    return hp.sigma / half_to_float(scales[g]);                 // sigma in weight units
+}
+
+// Eq. 4 (GATE) or saturation (CLAMP): the step actually applied to code w.
+long long applied_step(int w, long long step, int qmin, int qmax, int mode) {
+    long long target = (long long)w + step;
+    if (mode == 0) return (target >= qmin && target <= qmax) ? step : 0;
+    long long c = std::min<long long>(qmax, std::max<long long>(qmin, target));
+    return c - w;
+}
+
+int check(const Tensor& t, const HParams& hp) {
+    if (t.bits != 4 && t.bits != 8) return -2;
+    if (t.rows <= 0 || t.cols <= 0 || (t.cols & 1)) return -3;
+    if (t.group_size < 0 || (t.group_size > 0 && t.cols % t.group_size)) return -3;
+    if (!(hp.sigma > 0.f) || hp.n_pop <= 0 || !(hp.gamma >= 0.f && hp.gamma <= 1.f) || t.qmin >= t.qmax) return -5;
+    return 0;
+}
+
+template <class F> void parallel_for(int64_t n, int nthreads, F body) {
+    nthreads = std::max(1, nthreads);
+    if (nthreads == 1 || n < 2 * nthreads) { body((int64_t)0, n); return; }
+    std::vector<std::thread> th;
+    for (int w = 0; w < nthreads; ++w) {
+        int64_t lo = n * w / nthreads, hi = n * (w + 1) / nthreads;
+        th.emplace_back([=] { body(lo, hi); });
+    }
+    for (auto& x : th) x.join();
+}
+
+struct ElemResult { int w_new; double e_new; double band; int gate_final; int gate_replay; int attempted; };
+
+// Algorithm 2 for one element (Algorithm 1 when gens == 1 and e0 is the stored
+// residual).  gens generations, oldest first; the last one is the real update
+// unless replay_only.  Gating is always against the current code w (Sec. 3.3).
+ElemResult element_update(const Tensor& t, const HParams& hp, const uint16_t* scales, int w, int64_t j,
+                          const uint64_t* seeds, const float* fitness, int gens, double e0,
+                          bool replay_only, int tier) {
+    uint64_t J = t.elem_offset + (uint64_t)j;
+    uint64_t p = J >> 1;
+    int h = (int)(J & 1);
+    float sig[2];
+    sig[h] = sigma_eff(t, hp, scales, j);
+    sig[h ^ 1] = sig[h];
+    const int N = hp.n_pop;
+    const double c = (double)hp.lr / ((double)N * (double)hp.sigma);
+    const double gamma = (double)hp.gamma;
+    ElemResult r{w, e0, 0.5, 0, 0, 0};
+    double e = e0;
+    for (int k = 0; k < gens; ++k) {
+        double S = 0.0;
+        for (int i = 0; i < N; ++i) {
+            PairNoise pn = pair_noise(seeds[(int64_t)k * N + i], p, sig, tier, 0.0);
+            S += (double)fitness[(int64_t)k * N + i] * (double)pn.delta[h];   // Eq. 5 numerator
+        }
+        double u = c * S + gamma * e;                                          // Eq. 6
+        double step = std::round(u);                                           // Eq. 7, half away from zero
+        double dist = std::fabs(std::fabs(u - std::trunc(u)) - 0.5);
+        r.band = std::min(r.band, dist);
+        long long applied = applied_step(w, (long long)step, t.qmin, t.qmax, hp.boundary_mode);
+        bool blocked = applied != (long long)step;
+        e = u - (double)applied;                                               // Eq. 8 with the gated step
+        bool last = (k == gens - 1) && !replay_only;
+        if (last) {
+            r.w_new = w + (int)applied;
+            r.gate_final = blocked ? 1 : 0;
+            r.attempted = step != 0.0 ? 1 : 0;
+        } else if (blocked) {
+            r.gate_replay += 1;
+        }
+    }
+    r.e_new = e;
+    return r;
+}
+
+}  // namespace
+
+extern "C" {
+
+void qo_philox4x32_10(const uint32_t* ctr, const uint32_t* key, uint32_t* out) {
+    U4 r = philox4x32_10(ctr[0], ctr[1], ctr[2], ctr[3], key[0], key[1]);
+    std::memcpy(out, r.v, 16);
+}
+
+// Tier-1 Box-Muller factors for word pairs (r0[i], r1[i]).
+void qo_bm24(const uint32_t* r0, const uint32_t* r1, int64_t n, float* R, float* C, float* S) {
+    for (int64_t i = 0; i < n; ++i) {
+        R[i] = bm24_radius(r0[i]);
+        bm24_cossin(r1[i], &C[i], &S[i]);
+    }
+}
+
+int qo_stochastic_round(float x, uint32_t rword) { return stochastic_round_f32(x, rword); }
+
+float qo_half_to_float(uint16_t h) { return half_to_float(h); }
+
+// delta (and optionally x = sigma_eff * eps, near-decision flags) of global
+// elements J[0..n) for one seed and one sigma_eff.
+void qo_delta(uint64_t seed, const uint64_t* J, int64_t n, float sigma_eff_v, int tier, double tau,
+              int32_t* delta, double* x, uint8_t* near) {
+    float sig[2] = {sigma_eff_v, sigma_eff_v};
+    for (int64_t i = 0; i < n; ++i) {
+        PairNoise pn = pair_noise(seed, J[i] >> 1, sig, tier, tau);
+        int h = (int)(J[i] & 1);
+        delta[i] = pn.delta[h];
+        if (x) x[i] = pn.x[h];
+        if (near) near[i] = pn.near[h] ? 1 : 0;
+    }
+}
+
+void qo_unpack(int bits, const uint8_t* packed, int64_t n, int32_t* codes) {
+    for (int64_t j = 0; j < n; ++j) codes[j] = load_code(packed, bits, j);
+}
+void qo_pack(int bits, const int32_t* codes, int64_t n, uint8_t* packed) {
+    for (int64_t j = 0; j < n; ++j) store_code(packed, bits, j, codes[j]);
+}
+long long qo_applied_step(int w, long long step, int qmin, int qmax, int mode) {
+    return applied_step(w, step, qmin, qmax, mode);
+}
+
+// Algorithm 1, lines "Reconstruct delta_i" and "Gate(W + delta_i)" for one member.
+// idx == NULL: elements 0..n-1.  w_out[i] = perturbed code of element idx[i].
+int qo_perturb(const Tensor* t, const uint8_t* w, const uint16_t* scales, uint64_t seed,
+               const HParams* hp, int tier, const int64_t* idx, int64_t n, int nthreads, int32_t* w_out) {
+    int rc = check(*t, *hp);
+    if (rc) return rc;
+    parallel_for(n, nthreads, [=](int64_t lo, int64_t hi) {
+        for (int64_t i = lo; i < hi; ++i) {
+            int64_t j = idx ? idx[i] : i;
+            uint64_t J = t->elem_offset + (uint64_t)j;
+            int h = (int)(J & 1);
+            float sig[2];
+            sig[0] = sig[1] = sigma_eff(*t, *hp, scales, j);
+            PairNoise pn = pair_noise(seed, J >> 1, sig, tier, 0.0);
+            int code = load_code(w, t->bits, j);
+            w_out[i] = code + (int)applied_step(code, pn.delta[h], t->qmin, t->qmax, hp->boundary_mode);
+        }
+    });
+    return 0;
+}
+
+// Stateless update (Algorithm 2): seeds/fitness hold K+1 generations, oldest
+// first, the last being the current one.  With residual_in != NULL, K must be
+// 0 and this is one step of Algorithm 1 with the stored residual.
+// Outputs (each nullable except w_new): new code, residual after the step,
+// smallest distance of any generation's u to a rounding boundary, whether the
+// final step was blocked, number of blocked replay steps, whether the final
+// rounded step was non-zero.
+int qo_update(const Tensor* t, const uint8_t* w, const uint16_t* scales, const uint64_t* seeds,
+              const float* fitness, int K, const float* residual_in, const HParams* hp, int tier,
+              const int64_t* idx, int64_t n, int nthreads,
+              int32_t* w_new, double* e_new, double* band, uint8_t* gate_final, int32_t* gate_replay,
+              uint8_t* attempted) {
+    int rc = check(*t, *hp);
+    if (rc) return rc;
+    if (K < 0) return -5;
+    if (residual_in && K != 0) return -6;
+    parallel_for(n, nthreads, [=](int64_t lo, int64_t hi) {
+        for (int64_t i = lo; i < hi; ++i) {
+            int64_t j = idx ? idx[i] : i;
+            int code = load_code(w, t->bits, j);
+            double e0 = residual_in ? (double)residual_in[j] : 0.0;
+            ElemResult r = element_update(*t, *hp, scales, code, j, seeds, fitness, K + 1, e0, false, tier);
+            w_new[i] = r.w_new;
+            if (e_new) e_new[i] = r.e_new;
+            if (band) band[i] = r.band;
+            if (gate_final) gate_final[i] = (uint8_t)r.gate_final;
+            if (gate_replay) gate_replay[i] = r.gate_replay;
+            if (attempted) attempted[i] = (uint8_t)r.attempted;
+        }
+    });
+    return 0;
+}
+
+// The history loop of Algorithm 2 alone: proxy residual after K generations.
+int qo_replay_residual(const Tensor* t, const uint8_t* w, const uint16_t* scales, const uint64_t* seeds,
+                       const float* fitness, int K, const HParams* hp, int tier,
+                       const int64_t* idx, int64_t n, int nthreads,
+                       double* e_out, double* band, int32_t* gate_replay) {
+    int rc = check(*t, *hp);
+    if (rc) return rc;
+    if (K < 0) return -5;
+    parallel_for(n, nthreads, [=](int64_t lo, int64_t hi) {
+        for (int64_t i = lo; i < hi; ++i) {
+            int64_t j = idx ? idx[i] : i;
+            int code = load_code(w, t->bits, j);
+            ElemResult r = element_update(*t, *hp, scales, code, j, seeds, fitness, K, 0.0, true, tier);
+            e_out[i] = r.e_new;
+            if (band) band[i] = r.band;
+            if (gate_replay) gate_replay[i] = r.gate_replay;
+        }
+    });
+    return 0;
+}
+
+}  // extern "C"
