@@ -1,0 +1,125 @@
+/*
+ * libqes — the per-iteration parameter pass of Quantized Evolution Strategies (QES) on one GPU.
+ *
+ * Three operations over a packed low-bit weight tensor, every noise sample regenerated in
+ * registers from integer seeds (nothing but the weights is ever stored):
+ *   qes_perturb          W' = Gate(W + delta_i)                     Algorithm 1, member loop; Eqs. 3-4
+ *   qes_update           reward-weighted sum, error feedback, round,
+ *                        gate, repack — with Stateless Seed Replay     Algorithm 2; Eqs. 5-8
+ *                        or with a stored residual                     Algorithm 1, update lines
+ *   qes_replay_residual  the history loop of Algorithm 2 alone        Sec. 3.3
+ *
+ * Conventions shared by all entry points
+ *  - Pointers named w*, scales*, seeds, fitness, residual*, stats are DEVICE pointers owned by the
+ *    caller; the two structs are HOST pointers read during the call.  The library allocates
+ *    nothing, keeps no state between calls, enqueues its kernel on `cuda_stream` (a cudaStream_t
+ *    passed as void*; NULL = the legacy default stream) and returns without synchronising.
+ *  - Weights: row-major [rows, cols].  bits == 4: two codes per byte, even column in the low
+ *    nibble, two's complement; bits == 8: one signed byte per code.  The base address must be
+ *    16-byte aligned and rows*cols a multiple of 32 (one 128-bit word of INT4 codes).
+ *  - Scales: IEEE binary16, [rows, cols / group_size] row-major, or [rows] when group_size == 0.
+ *    Read only when sigma_unit == QES_SIGMA_WEIGHT; may be NULL otherwise.
+ *  - Noise: delta(seed, J) for global element index J = elem_offset + row*cols + col is
+ *    Philox4x32-10(key = seed, counter = J >> 1) -> Box-Muller -> sigma scaling -> stochastic
+ *    rounding (Eq. 3), limited to the 4-bit range [-8, 7] (App. A).  Results depend only on
+ *    (seed, J): any split of a model into tensors, any grid size, gives the same bits.
+ *  - Fitness values are the already normalised rewards F_i (Algorithm 1, "Normalize reward").
+ *  - Return value: QES_OK, or a negative qes_status; on any error nothing was launched and no
+ *    buffer was touched.
+ */
+#ifndef QES_H_
+#define QES_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    QES_OK = 0,
+    QES_ERR_NULL_PTR = -1,    /* a required pointer is NULL */
+    QES_ERR_BAD_BITS = -2,    /* bits is not 4 or 8 */
+    QES_ERR_BAD_SHAPE = -3,   /* rows/cols/group_size/elem_offset violate the layout rules */
+    QES_ERR_MISALIGNED = -4,  /* a device pointer misses its alignment (16 B weights/residual, 8 B seeds, 4 B fitness, 2 B scales) */
+    QES_ERR_BAD_HPARAM = -5,  /* sigma <= 0, n_pop <= 0, K < 0, gamma outside [0,1], qmin >= qmax, range outside the code width */
+    QES_ERR_BAD_MODE = -6,    /* unknown sigma_unit / boundary_mode, or residual_inout given with K > 0 */
+    QES_ERR_CUDA = -7,        /* the launch reported a CUDA error (cudaGetLastError) */
+    QES_ERR_TOO_LARGE = -8    /* the (K+1)*n_pop table does not fit the kernel's shared-memory staging */
+} qes_status;
+
+enum { QES_SIGMA_GRID = 0, QES_SIGMA_WEIGHT = 1 };   /* unit of hparams.sigma: grid steps | weight units (sigma_g = sigma / scale_g) */
+enum { QES_BOUNDARY_GATE = 0, QES_BOUNDARY_CLAMP = 1 }; /* Eq. 4 masking | saturation */
+
+typedef struct {
+    int32_t bits;          /* 4 or 8 */
+    int32_t qmin, qmax;    /* inclusive code range, e.g. -8..7, -7..7 (App. A grid), -128..127 */
+    int32_t group_size;    /* codes per scale along a row (multiple of 32); 0 = one scale per row */
+    int64_t rows, cols;    /* cols % 32 == 0; cols % group_size == 0 */
+    uint64_t elem_offset;  /* global index of element (0,0); multiple of 32 */
+} qes_tensor_desc;
+
+typedef struct {
+    float sigma;           /* perturbation scale sigma of Eq. 3 (> 0) */
+    float lr;              /* learning rate alpha of Eq. 6 */
+    float gamma;           /* residual decay gamma of Eq. 6, in [0, 1] */
+    int32_t n_pop;         /* population size N */
+    int32_t sigma_unit;    /* QES_SIGMA_GRID | QES_SIGMA_WEIGHT */
+    int32_t boundary_mode; /* QES_BOUNDARY_GATE | QES_BOUNDARY_CLAMP */
+} qes_hparams;
+
+/*
+ * Algorithm 1, "Reconstruct delta_i" + "Gate(W_t + delta_i)" (Eqs. 3-4) for one population member.
+ *   w_in  [device, rows*cols codes]  current weights, not modified (unless w_out == w_in)
+ *   w_out [device, same size]        perturbed weights; may alias w_in exactly, no partial overlap
+ *   seed                             the member's seed s_i
+ * Only sigma, sigma_unit and boundary_mode of hparams are used (n_pop, lr, gamma still validated).
+ */
+int qes_perturb(const qes_tensor_desc* desc, const void* w_in, void* w_out, const void* scales_f16,
+                uint64_t seed, const qes_hparams* hparams, void* cuda_stream);
+
+/*
+ * Algorithm 2, history loop (proxy residual): for k = 0..K-1, u = alpha*g_k + gamma*e,
+ * Delta = Round(u), gated against the CURRENT weights w, e = u - Delta_final.
+ *   seeds   [device, K*n_pop uint64]  generation-major, oldest generation first
+ *   fitness [device, K*n_pop float]   same order
+ *   residual_out [device, rows*cols float]  e after the K generations (K == 0 writes zeros)
+ */
+int qes_replay_residual(const qes_tensor_desc* desc, const void* w, const void* scales_f16,
+                        const uint64_t* seeds, const float* fitness, int32_t K,
+                        const qes_hparams* hparams, float* residual_out, void* cuda_stream);
+
+/*
+ * The update.  residual_inout == NULL: stateless (Algorithm 2) — replays K history generations
+ * from e = 0, then applies the current generation; seeds/fitness hold K+1 generations, the last
+ * row being the current one.  residual_inout != NULL: stored residual (Algorithm 1, Eqs. 6-8) —
+ * K must be 0; e is read, and e_{t+1} = u - Delta_final written back (fp32).
+ *   w_inout [device]  updated in place: W <- W + Delta_final
+ *   stats   [device, 4 x uint64, nullable]  counters ADDED to (caller zeroes): [0] codes changed,
+ *           [1] final steps blocked or shortened by the boundary, [2] blocked replay steps,
+ *           [3] non-zero rounded final steps (before the boundary rule)
+ */
+int qes_update(const qes_tensor_desc* desc, void* w_inout, const void* scales_f16,
+               const uint64_t* seeds, const float* fitness, int32_t K, float* residual_inout,
+               const qes_hparams* hparams, uint64_t* stats, void* cuda_stream);
+
+/*
+ * Arithmetic-pipe throughput probes used to derive the ALU roofline (no counterpart in the
+ * paper).  Runs `iters` dependent-chain iterations of one instruction kind on every lane of a
+ * full grid and writes the elapsed device time in milliseconds to *ms_out (HOST pointer) and
+ * the number of lane-operations performed to *ops_out (HOST pointer).  sink_dev is a DEVICE
+ * buffer of at least 4 bytes owned by the caller (the probes keep their results live by a store
+ * that is practically never taken).  Runs on the default stream and synchronises.
+ *   kind: 0 mul.wide.u32  1 lop3 (xor3)  2 fma.rn.f32  3 mul.hi.u32  4 cvt.rn.f32.u32
+ *         5 sqrt.rn.f32   6 cvt.rmi (floor)  7 mad.lo.u32  8 Philox round (2 wide multiplies + 2 xor3)
+ *         9 rsqrt.approx.f32 (special-function unit)
+ */
+int qes_pipe_probe(int32_t kind, int32_t iters, void* sink_dev, float* ms_out, double* ops_out);
+
+const char* qes_strerror(int status);
+int qes_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QES_H_ */

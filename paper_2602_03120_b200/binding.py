@@ -1,0 +1,188 @@
+"""Thin ctypes binding of ``libqes.so``: argument marshalling only.
+
+Every step of the parameter pass runs inside the CUDA kernels of the library; this module turns
+torch CUDA tensors into device pointers, fills the two C structs and raises on error codes.  It
+never falls back to another implementation: a missing library is an ImportError-like failure.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libqes.so")
+
+SIGMA_GRID, SIGMA_WEIGHT = 0, 1
+BOUNDARY_GATE, BOUNDARY_CLAMP = 0, 1
+
+
+class QesError(RuntimeError):
+    pass
+
+
+class _TensorDesc(C.Structure):
+    _fields_ = [("bits", C.c_int32), ("qmin", C.c_int32), ("qmax", C.c_int32), ("group_size", C.c_int32),
+                ("rows", C.c_int64), ("cols", C.c_int64), ("elem_offset", C.c_uint64)]
+
+
+class _HParams(C.Structure):
+    _fields_ = [("sigma", C.c_float), ("lr", C.c_float), ("gamma", C.c_float),
+                ("n_pop", C.c_int32), ("sigma_unit", C.c_int32), ("boundary_mode", C.c_int32)]
+
+
+@dataclass
+class TensorDesc:
+    bits: int
+    rows: int
+    cols: int
+    qmin: int | None = None
+    qmax: int | None = None
+    group_size: int = 0
+    elem_offset: int = 0
+
+    def c(self) -> _TensorDesc:
+        qmin = -(1 << (self.bits - 1)) if self.qmin is None else self.qmin
+        qmax = (1 << (self.bits - 1)) - 1 if self.qmax is None else self.qmax
+        return _TensorDesc(self.bits, qmin, qmax, self.group_size, self.rows, self.cols, self.elem_offset)
+
+    @property
+    def numel(self) -> int:
+        return self.rows * self.cols
+
+    @property
+    def packed_bytes(self) -> int:
+        return self.numel if self.bits == 8 else self.numel // 2
+
+
+@dataclass
+class HParams:
+    sigma: float
+    lr: float
+    gamma: float
+    n_pop: int
+    sigma_unit: int = SIGMA_GRID
+    boundary_mode: int = BOUNDARY_GATE
+
+    def c(self) -> _HParams:
+        return _HParams(self.sigma, self.lr, self.gamma, self.n_pop, self.sigma_unit, self.boundary_mode)
+
+
+_lib = None
+
+
+def load() -> C.CDLL:
+    """Load the compiled library; raises if it has not been built (there is no other code path)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise QesError(f"{LIB_PATH} is missing: run paper_2602_03120_b200.build.build_library() "
+                           "(nvcc, sm_100a); the parameter pass has no fallback implementation")
+        lib = C.CDLL(LIB_PATH)
+        vp, u64, i32 = C.c_void_p, C.c_uint64, C.c_int32
+        lib.qes_perturb.restype = C.c_int
+        lib.qes_perturb.argtypes = [C.POINTER(_TensorDesc), vp, vp, vp, u64, C.POINTER(_HParams), vp]
+        lib.qes_replay_residual.restype = C.c_int
+        lib.qes_replay_residual.argtypes = [C.POINTER(_TensorDesc), vp, vp, vp, vp, i32, C.POINTER(_HParams), vp, vp]
+        lib.qes_update.restype = C.c_int
+        lib.qes_update.argtypes = [C.POINTER(_TensorDesc), vp, vp, vp, vp, i32, vp, C.POINTER(_HParams), vp, vp]
+        lib.qes_pipe_probe.restype = C.c_int
+        lib.qes_pipe_probe.argtypes = [i32, i32, vp, C.POINTER(C.c_float), C.POINTER(C.c_double)]
+        lib.qes_strerror.restype = C.c_char_p
+        lib.qes_strerror.argtypes = [C.c_int]
+        lib.qes_version.restype = C.c_int
+        _lib = lib
+    return _lib
+
+
+def _ptr(t, *, dtype=None, nbytes=None, name="tensor"):
+    if t is None:
+        return None
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise QesError(f"{name} must be a CUDA tensor")
+    if not t.is_contiguous():
+        raise QesError(f"{name} must be contiguous")
+    if dtype is not None and t.dtype not in (dtype if isinstance(dtype, tuple) else (dtype,)):
+        raise QesError(f"{name} has dtype {t.dtype}, expected {dtype}")
+    if nbytes is not None and t.numel() * t.element_size() < nbytes:
+        raise QesError(f"{name} holds {t.numel() * t.element_size()} bytes, needs {nbytes}")
+    return t.data_ptr()
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def _check(rc: int):
+    if rc != 0:
+        raise QesError(f"libqes error {rc}: {load().qes_strerror(rc).decode()}")
+
+
+_W = (torch.uint8, torch.int8)
+_S = (torch.float16,)
+_SEEDS = (torch.int64, torch.uint64)
+
+
+def _scale_bytes(d: TensorDesc) -> int:
+    return 2 * (d.rows * (d.cols // d.group_size) if d.group_size else d.rows)
+
+
+def qes_perturb(desc: TensorDesc, w_in, w_out, scales_f16, seed: int, hparams: HParams, stream=None) -> None:
+    """W' = Gate(W + delta_i) for one member (Algorithm 1; Eqs. 3-4).  Enqueues, does not synchronise."""
+    d, h = desc.c(), hparams.c()
+    rc = load().qes_perturb(C.byref(d), _ptr(w_in, dtype=_W, nbytes=desc.packed_bytes, name="w_in"),
+                            _ptr(w_out, dtype=_W, nbytes=desc.packed_bytes, name="w_out"),
+                            _ptr(scales_f16, dtype=_S, nbytes=_scale_bytes(desc), name="scales"),
+                            C.c_uint64(seed & 0xFFFFFFFFFFFFFFFF), C.byref(h), _stream(stream))
+    _check(rc)
+
+
+def qes_replay_residual(desc: TensorDesc, w, scales_f16, seeds, fitness, K: int, hparams: HParams,
+                        residual_out, stream=None) -> None:
+    """History loop of Algorithm 2: writes the proxy residual after K generations (fp32)."""
+    d, h = desc.c(), hparams.c()
+    n = K * hparams.n_pop
+    rc = load().qes_replay_residual(C.byref(d), _ptr(w, dtype=_W, nbytes=desc.packed_bytes, name="w"),
+                                    _ptr(scales_f16, dtype=_S, nbytes=_scale_bytes(desc), name="scales"),
+                                    _ptr(seeds, dtype=_SEEDS, nbytes=8 * n, name="seeds"),
+                                    _ptr(fitness, dtype=torch.float32, nbytes=4 * n, name="fitness"),
+                                    K, C.byref(h),
+                                    _ptr(residual_out, dtype=torch.float32, nbytes=4 * desc.numel, name="residual_out"),
+                                    _stream(stream))
+    _check(rc)
+
+
+def qes_update(desc: TensorDesc, w_inout, scales_f16, seeds, fitness, K: int, residual_inout,
+               hparams: HParams, stats=None, stream=None) -> None:
+    """In-place update: stateless with seed replay (Algorithm 2) or with a stored residual (Algorithm 1)."""
+    d, h = desc.c(), hparams.c()
+    n = (K + 1) * hparams.n_pop
+    rc = load().qes_update(C.byref(d), _ptr(w_inout, dtype=_W, nbytes=desc.packed_bytes, name="w_inout"),
+                           _ptr(scales_f16, dtype=_S, nbytes=_scale_bytes(desc), name="scales"),
+                           _ptr(seeds, dtype=_SEEDS, nbytes=8 * n, name="seeds"),
+                           _ptr(fitness, dtype=torch.float32, nbytes=4 * n, name="fitness"),
+                           K, _ptr(residual_inout, dtype=torch.float32, nbytes=4 * desc.numel, name="residual_inout"),
+                           C.byref(h), _ptr(stats, dtype=_SEEDS, nbytes=32, name="stats"), _stream(stream))
+    _check(rc)
+
+
+PROBE_KINDS = {0: "mul.wide.u32", 1: "lop3.xor3", 2: "fma.rn.f32", 3: "mul.hi.u32", 4: "cvt.rn.f32.u32",
+               5: "sqrt.rn.f32", 6: "cvt.rmi.f32.f32", 7: "mad.lo.u32", 8: "philox round (2 mul.wide + 2 xor3)",
+               9: "rsqrt.approx.f32", 10: "add.u32", 11: "shr.u32", 12: "add.rn.f32", 13: "mul.rn.f32",
+               14: "setp.lt.f32 + selp", 15: "min.f32", 16: "cvt.rzi.s32.f32", 17: "set.lt.f32 (1.0/0.0)",
+               100: "mix mul.wide + xor3", 101: "mix fma + xor3", 102: "mix mul.wide + fma", 103: "mix cvt.f32.u32 + xor3",
+               104: "mix cvt.f32.u32 + mul.wide", 105: "mix floor + rsqrt", 106: "mix floor + fma", 107: "mix add + xor3",
+               108: "mix fadd + mul.wide", 109: "mix setp/selp + fma"}
+
+
+def qes_pipe_probe(kind: int, iters: int = 4096):
+    """Lane-operations per second of one instruction kind on the current device (synchronises)."""
+    sink = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ms, ops = C.c_float(0), C.c_double(0)
+    torch.cuda.synchronize()
+    _check(load().qes_pipe_probe(kind, iters, sink.data_ptr(), C.byref(ms), C.byref(ops)))
+    return ops.value / (ms.value * 1e-3), ms.value

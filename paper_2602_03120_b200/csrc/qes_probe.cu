@@ -1,0 +1,209 @@
+// Arithmetic-pipe throughput probes: the measured denominators of the ALU roofline.
+// Each probe runs kChains independent dependent-chains of one PTX instruction per thread on a
+// grid that fills every SM, and reports lane-operations and elapsed device time.
+#include <cstdint>
+#include <cuda_runtime.h>
+#include "../../include/qes.h"
+
+namespace {
+
+constexpr int kChains = 8;
+constexpr int kProbeThreads = 256;
+constexpr int kCtasPerSm = 8;
+
+template <int KIND>
+__device__ __forceinline__ uint32_t step(uint32_t x, uint32_t a, uint32_t b) {
+    uint32_t r;
+    if (KIND == 0) {          // 32x32 -> 64 multiply, low word carried
+        unsigned long long w;
+        asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(w) : "r"(x), "r"(a));
+        r = (uint32_t)w ^ 0u;
+        asm volatile("" : "+r"(r));
+    } else if (KIND == 1) {   // three-input xor
+        asm volatile("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(r) : "r"(x), "r"(a), "r"(b));
+    } else if (KIND == 2) {   // fp32 fused multiply-add
+        float f;
+        asm volatile("fma.rn.f32 %0, %1, %2, %3;" : "=f"(f) : "f"(__uint_as_float(x)), "f"(__uint_as_float(a)), "f"(__uint_as_float(b)));
+        r = __float_as_uint(f);
+    } else if (KIND == 3) {   // high half of 32x32 multiply
+        asm volatile("mul.hi.u32 %0, %1, %2;" : "=r"(r) : "r"(x), "r"(a));
+    } else if (KIND == 4) {   // unsigned -> float conversion
+        float f;
+        asm volatile("cvt.rn.f32.u32 %0, %1;" : "=f"(f) : "r"(x));
+        r = __float_as_uint(f);
+    } else if (KIND == 5) {   // correctly rounded square root
+        float f;
+        asm volatile("sqrt.rn.f32 %0, %1;" : "=f"(f) : "f"(__uint_as_float(x)));
+        r = __float_as_uint(f);
+    } else if (KIND == 6) {   // floor
+        float f;
+        asm volatile("cvt.rmi.f32.f32 %0, %1;" : "=f"(f) : "f"(__uint_as_float(x)));
+        r = __float_as_uint(f);
+    } else if (KIND == 7) {   // 32-bit multiply-add
+        asm volatile("mad.lo.u32 %0, %1, %2, %3;" : "=r"(r) : "r"(x), "r"(a), "r"(b));
+    } else if (KIND == 9) {   // special-function unit
+        float f;
+        asm volatile("rsqrt.approx.f32 %0, %1;" : "=f"(f) : "f"(__uint_as_float(x)));
+        r = __float_as_uint(f);
+    } else if (KIND == 10) {  // integer add
+        asm volatile("add.u32 %0, %1, %2;" : "=r"(r) : "r"(x), "r"(a));
+    } else if (KIND == 11) {  // funnel/logical shift
+        asm volatile("shr.u32 %0, %1, 1;" : "=r"(r) : "r"(x));
+        asm volatile("" : "+r"(r));
+    } else if (KIND == 12) {  // fp32 add
+        float f;
+        asm volatile("add.rn.f32 %0, %1, %2;" : "=f"(f) : "f"(__uint_as_float(x)), "f"(__uint_as_float(b)));
+        r = __float_as_uint(f);
+    } else if (KIND == 13) {  // fp32 multiply
+        float f;
+        asm volatile("mul.rn.f32 %0, %1, %2;" : "=f"(f) : "f"(__uint_as_float(x)), "f"(__uint_as_float(b)));
+        r = __float_as_uint(f);
+    } else if (KIND == 14) {  // fp32 compare + select
+        asm volatile("{ .reg .pred p; setp.lt.f32 p, %1, %2; selp.b32 %0, %3, %1, p; }" : "=r"(r) : "r"(x), "r"(b), "r"(a));
+    } else if (KIND == 15) {  // fp32 min
+        float f;
+        asm volatile("min.f32 %0, %1, %2;" : "=f"(f) : "f"(__uint_as_float(x)), "f"(__uint_as_float(b)));
+        r = __float_as_uint(f);
+    } else if (KIND == 16) {  // float -> int conversion
+        asm volatile("cvt.rzi.s32.f32 %0, %1;" : "=r"(r) : "f"(__uint_as_float(x)));
+    } else if (KIND == 17) {  // compare to 1.0f/0.0f
+        float f;
+        asm volatile("set.lt.f32.f32 %0, %1, %2;" : "=f"(f) : "f"(__uint_as_float(x)), "f"(__uint_as_float(b)));
+        r = __float_as_uint(f);
+    } else {
+        r = x;
+    }
+    return r;
+}
+
+template <int KIND>
+__global__ void __launch_bounds__(kProbeThreads) probe_kernel(int iters, uint32_t a, uint32_t b, uint32_t* sink) {
+    uint32_t x[kChains];
+#pragma unroll
+    for (int c = 0; c < kChains; ++c) x[c] = threadIdx.x * 2654435761u + c * 40503u + blockIdx.x + 0x3f800001u;
+    if (KIND == 8) {
+        // one Philox round per chain pair: 2 wide multiplies + 2 three-input xors per 4 words
+        for (int it = 0; it < iters; ++it) {
+#pragma unroll
+            for (int c = 0; c < kChains; c += 4) {
+                unsigned long long p0 = (unsigned long long)0xD2511F53u * x[c];
+                unsigned long long p1 = (unsigned long long)0xCD9E8D57u * x[c + 2];
+                uint32_t n0 = (uint32_t)(p1 >> 32) ^ x[c + 1] ^ a;
+                uint32_t n2 = (uint32_t)(p0 >> 32) ^ x[c + 3] ^ b;
+                x[c + 1] = (uint32_t)p1; x[c + 3] = (uint32_t)p0; x[c] = n0; x[c + 2] = n2;
+            }
+            a += 0x9E3779B9u; b += 0xBB67AE85u;
+        }
+    } else {
+        for (int it = 0; it < iters; ++it) {
+#pragma unroll
+            for (int c = 0; c < kChains; ++c) x[c] = step<KIND>(x[c], a, b);
+        }
+    }
+    uint32_t acc = 0;
+#pragma unroll
+    for (int c = 0; c < kChains; ++c) acc ^= x[c];
+    if (acc == 0x12345u) sink[0] = acc;   // keeps the chains live; practically never taken
+}
+
+template <int KA, int KB>
+__global__ void __launch_bounds__(kProbeThreads) probe_mix_kernel(int iters, uint32_t a, uint32_t b, uint32_t* sink) {
+    uint32_t x[kChains];
+#pragma unroll
+    for (int c = 0; c < kChains; ++c) x[c] = threadIdx.x * 2654435761u + c * 40503u + blockIdx.x + 0x3f800001u;
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int c = 0; c < kChains; c += 2) {
+            x[c] = step<KA>(x[c], a, b);
+            x[c + 1] = step<KB>(x[c + 1], a, b);
+        }
+    }
+    uint32_t acc = 0;
+#pragma unroll
+    for (int c = 0; c < kChains; ++c) acc ^= x[c];
+    if (acc == 0x12345u) sink[0] = acc;
+}
+
+template <int KA, int KB>
+int run_mix(int iters, uint32_t* sink, float* ms_out, double* ops_out) {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return QES_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return QES_ERR_CUDA;
+    cudaEvent_t e0, e1;
+    cudaEventCreate(&e0); cudaEventCreate(&e1);
+    int blocks = sms * kCtasPerSm;
+    probe_mix_kernel<KA, KB><<<blocks, kProbeThreads>>>(iters / 8 + 1, 0x9E3779B9u, 0x3f7ffff0u, sink);
+    cudaEventRecord(e0);
+    probe_mix_kernel<KA, KB><<<blocks, kProbeThreads>>>(iters, 0x9E3779B9u, 0x3f7ffff0u, sink);
+    cudaEventRecord(e1);
+    cudaError_t err = cudaEventSynchronize(e1);
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, e0, e1);
+    cudaEventDestroy(e0); cudaEventDestroy(e1);
+    if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return QES_ERR_CUDA;
+    *ms_out = ms;
+    *ops_out = (double)blocks * kProbeThreads * (double)iters * (double)kChains;
+    return QES_OK;
+}
+
+template <int KIND>
+int run_probe(int iters, uint32_t* sink, float* ms_out, double* ops_out) {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return QES_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return QES_ERR_CUDA;
+    cudaEvent_t e0, e1;
+    cudaEventCreate(&e0); cudaEventCreate(&e1);
+    int blocks = sms * kCtasPerSm;
+    probe_kernel<KIND><<<blocks, kProbeThreads>>>(iters / 8 + 1, 0x9E3779B9u, 0x3f7ffff0u, sink);   // warm-up
+    cudaEventRecord(e0);
+    probe_kernel<KIND><<<blocks, kProbeThreads>>>(iters, 0x9E3779B9u, 0x3f7ffff0u, sink);
+    cudaEventRecord(e1);
+    cudaError_t err = cudaEventSynchronize(e1);
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, e0, e1);
+    cudaEventDestroy(e0); cudaEventDestroy(e1);
+    if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return QES_ERR_CUDA;
+    *ms_out = ms;
+    double per_iter = (KIND == 8) ? (kChains / 4) * 4.0 : (double)kChains;   // kind 8: 4 instructions per 4-word round
+    *ops_out = (double)blocks * kProbeThreads * (double)iters * per_iter;
+    return QES_OK;
+}
+
+}  // namespace
+
+extern "C" int qes_pipe_probe(int32_t kind, int32_t iters, void* sink_dev, float* ms_out, double* ops_out) {
+    if (ms_out == nullptr || ops_out == nullptr || sink_dev == nullptr) return QES_ERR_NULL_PTR;
+    uint32_t* sink = reinterpret_cast<uint32_t*>(sink_dev);
+    if (iters <= 0 || iters > (1 << 24)) return QES_ERR_BAD_HPARAM;
+    switch (kind) {
+        case 0: return run_probe<0>(iters, sink, ms_out, ops_out);
+        case 1: return run_probe<1>(iters, sink, ms_out, ops_out);
+        case 2: return run_probe<2>(iters, sink, ms_out, ops_out);
+        case 3: return run_probe<3>(iters, sink, ms_out, ops_out);
+        case 4: return run_probe<4>(iters, sink, ms_out, ops_out);
+        case 5: return run_probe<5>(iters, sink, ms_out, ops_out);
+        case 6: return run_probe<6>(iters, sink, ms_out, ops_out);
+        case 7: return run_probe<7>(iters, sink, ms_out, ops_out);
+        case 8: return run_probe<8>(iters, sink, ms_out, ops_out);
+        case 9: return run_probe<9>(iters, sink, ms_out, ops_out);
+        case 10: return run_probe<10>(iters, sink, ms_out, ops_out);
+        case 11: return run_probe<11>(iters, sink, ms_out, ops_out);
+        case 12: return run_probe<12>(iters, sink, ms_out, ops_out);
+        case 13: return run_probe<13>(iters, sink, ms_out, ops_out);
+        case 14: return run_probe<14>(iters, sink, ms_out, ops_out);
+        case 15: return run_probe<15>(iters, sink, ms_out, ops_out);
+        case 16: return run_probe<16>(iters, sink, ms_out, ops_out);
+        case 17: return run_probe<17>(iters, sink, ms_out, ops_out);
+        case 100: return run_mix<0, 1>(iters, sink, ms_out, ops_out);    // mul.wide + xor3
+        case 101: return run_mix<2, 1>(iters, sink, ms_out, ops_out);    // fma + xor3
+        case 102: return run_mix<0, 2>(iters, sink, ms_out, ops_out);    // mul.wide + fma
+        case 103: return run_mix<4, 1>(iters, sink, ms_out, ops_out);    // cvt + xor3
+        case 104: return run_mix<4, 0>(iters, sink, ms_out, ops_out);    // cvt + mul.wide
+        case 105: return run_mix<6, 9>(iters, sink, ms_out, ops_out);    // floor + rsqrt
+        case 106: return run_mix<6, 2>(iters, sink, ms_out, ops_out);    // floor + fma
+        case 107: return run_mix<10, 1>(iters, sink, ms_out, ops_out);   // add + xor3
+        case 108: return run_mix<12, 0>(iters, sink, ms_out, ops_out);   // fadd + mul.wide
+        case 109: return run_mix<14, 2>(iters, sink, ms_out, ops_out);   // compare/select + fma
+        default: return QES_ERR_BAD_MODE;
+    }
+}

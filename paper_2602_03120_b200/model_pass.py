@@ -1,0 +1,78 @@
+"""A whole weight set on one GPU: flat packed buffer, per-tensor descriptors, and the three passes.
+
+This is the call a user of the library makes for a model: ``perturb_member`` (Algorithm 1, member
+loop), ``update`` (Algorithm 2) and ``replay_residual`` launch one library call per tensor on the
+current stream.  Nothing here computes: every step runs in the kernels behind the C ABI.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import binding as qes
+from . import workloads as wl
+
+
+def shard_tensors(workload: wl.Workload, rank: int, world: int):
+    """Weak-scaling shard: rank r owns copy r of the decoder stack of a `world`-times deeper model.
+    Global element offsets continue across ranks, so every rank draws a disjoint noise stream and the
+    union equals one model of world*layers layers updated on one device.  No data is exchanged."""
+    per_rank = workload.numel
+    return tuple(wl.TensorSpec(f"shard{rank}.{t.name}", t.rows, t.cols, t.elem_offset + rank * per_rank)
+                 for t in workload.tensors)
+
+
+class ModelPass:
+    def __init__(self, workload: wl.Workload, device="cuda", rank: int = 0, world: int = 1,
+                 sigma_unit: int = qes.SIGMA_GRID, with_scales: bool = False):
+        self.wl = workload
+        self.device = torch.device(device)
+        self.tensors = shard_tensors(workload, rank, world)
+        self.base = self.tensors[0].elem_offset
+        self.numel = sum(t.numel for t in self.tensors)
+        self.bytes = wl.packed_bytes(workload.bits, self.numel)
+        self.w = torch.empty(self.bytes, dtype=torch.uint8, device=self.device)
+        self.hp = qes.HParams(sigma=workload.sigma, lr=workload.lr, gamma=workload.gamma, n_pop=workload.n_pop,
+                              sigma_unit=sigma_unit)
+        self.descs = [qes.TensorDesc(bits=workload.bits, rows=t.rows, cols=t.cols, group_size=workload.group_size,
+                                     elem_offset=t.elem_offset) for t in self.tensors]
+        self.scales = None
+        if with_scales or sigma_unit == qes.SIGMA_WEIGHT:
+            self.scales = [torch.from_numpy(wl.draw_scales(workload, i)).to(self.device)
+                           for i in range(len(self.tensors))]
+
+    def _slice(self, buf, t):
+        lo = wl.packed_bytes(self.wl.bits, t.elem_offset - self.base)
+        return buf[lo:lo + wl.packed_bytes(self.wl.bits, t.numel)]
+
+    def host_codes(self) -> np.ndarray:
+        """Packed synthetic codes of this shard on the host (uniform random bytes per tensor)."""
+        out = np.empty(self.bytes, np.uint8)
+        for i, t in enumerate(self.tensors):
+            lo = wl.packed_bytes(self.wl.bits, t.elem_offset - self.base)
+            out[lo:lo + wl.packed_bytes(self.wl.bits, t.numel)] = wl.draw_codes(self.wl, i)
+        return out
+
+    def load(self, host_packed) -> None:
+        self.w.copy_(host_packed if isinstance(host_packed, torch.Tensor) else torch.from_numpy(host_packed),
+                     non_blocking=True)
+
+    def _sc(self, i):
+        return None if self.scales is None else self.scales[i]
+
+    def perturb_member(self, out: torch.Tensor, seed: int) -> int:
+        for i, (t, d) in enumerate(zip(self.tensors, self.descs)):
+            qes.qes_perturb(d, self._slice(self.w, t), self._slice(out, t), self._sc(i), seed, self.hp)
+        return len(self.tensors)
+
+    def update(self, seeds: torch.Tensor, fitness: torch.Tensor, K: int, stats=None) -> int:
+        for i, (t, d) in enumerate(zip(self.tensors, self.descs)):
+            qes.qes_update(d, self._slice(self.w, t), self._sc(i), seeds, fitness, K, None, self.hp, stats=stats)
+        return len(self.tensors)
+
+    def replay_residual(self, seeds: torch.Tensor, fitness: torch.Tensor, K: int, out: torch.Tensor) -> int:
+        for i, (t, d) in enumerate(zip(self.tensors, self.descs)):
+            lo = t.elem_offset - self.base
+            qes.qes_replay_residual(d, self._slice(self.w, t), self._sc(i), seeds, fitness, K, self.hp,
+                                    out[lo:lo + t.numel])
+        return len(self.tensors)

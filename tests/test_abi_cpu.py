@@ -1,0 +1,71 @@
+"""CPU-side checks of the C ABI: the library loads, exports what the header declares, and turns
+invalid arguments into error codes before anything is launched (no GPU needed for any of it)."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2602_03120_b200 import binding, build
+    build.build_library()
+    return binding.load()
+
+
+def test_every_declared_symbol_is_exported(lib):
+    header = open(os.path.join(ROOT, "include", "qes.h")).read()
+    names = re.findall(r"^(?:int|const char\*)\s+(qes_\w+)\s*\(", header, flags=re.M)
+    assert set(names) >= {"qes_perturb", "qes_update", "qes_replay_residual", "qes_strerror", "qes_version"}
+    for n in names:
+        assert hasattr(lib, n), n
+    assert lib.qes_version() >= 100
+
+
+def test_struct_layouts_match_header():
+    from paper_2602_03120_b200 import binding
+    assert C.sizeof(binding._TensorDesc) == 40 and C.sizeof(binding._HParams) == 24
+    assert binding._TensorDesc.rows.offset == 16 and binding._TensorDesc.elem_offset.offset == 32
+
+
+def _call_update(lib, binding, *, bits=4, rows=4, cols=64, group=0, off=0, qmin=None, qmax=None,
+                 sigma=0.5, gamma=0.9, n_pop=4, K=1, w=0x1000, seeds=0x2000, fit=0x3000, res=None,
+                 unit=0, mode=0, scales=None):
+    d = binding.TensorDesc(bits=bits, rows=rows, cols=cols, group_size=group, elem_offset=off, qmin=qmin, qmax=qmax).c()
+    h = binding.HParams(sigma=sigma, lr=1.0, gamma=gamma, n_pop=n_pop, sigma_unit=unit, boundary_mode=mode).c()
+    return lib.qes_update(C.byref(d), w, scales, seeds, fit, K, res, C.byref(h), None, None)
+
+
+def test_invalid_arguments_are_rejected_without_launching(lib):
+    from paper_2602_03120_b200 import binding
+    call = lambda **kw: _call_update(lib, binding, **kw)
+    assert call(bits=5) == -2
+    assert call(cols=48) == -3 and call(rows=0) == -3 and call(group=48) == -3 and call(cols=64, group=128) == -3
+    assert call(off=16) == -3
+    assert call(w=0x1008) == -4 and call(seeds=0x2004) == -4 and call(res=0x4004, K=0) == -4
+    assert call(sigma=0.0) == -5 and call(sigma=-1.0) == -5 and call(n_pop=0) == -5 and call(K=-1) == -5
+    assert call(gamma=1.5) == -5 and call(qmin=3, qmax=3) == -5 and call(qmin=-9, qmax=7) == -5
+    assert call(unit=2) == -6 and call(mode=7) == -6 and call(res=0x4000, K=2) == -6
+    assert call(w=None) == -1 and call(seeds=None) == -1 and call(unit=1, scales=None) == -1
+    assert call(n_pop=1000, K=100) == -8
+    d = binding.TensorDesc(bits=4, rows=4, cols=64).c()
+    h = binding.HParams(sigma=0.5, lr=1.0, gamma=0.9, n_pop=4).c()
+    assert lib.qes_perturb(C.byref(d), None, 0x1000, None, 1, C.byref(h), None) == -1
+    assert lib.qes_perturb(None, 0x1000, 0x1000, None, 1, C.byref(h), None) == -1
+    assert lib.qes_replay_residual(C.byref(d), 0x1000, None, 0x2000, 0x3000, 2, C.byref(h), None, None) == -1
+    assert lib.qes_replay_residual(C.byref(d), 0x1000, None, 0x2000, 0x3000, 2, C.byref(h), 0x4008, None) == -4
+    for code in range(-8, 1):
+        assert len(lib.qes_strerror(code)) > 1
+
+
+def test_binding_refuses_host_tensors():
+    import torch
+    from paper_2602_03120_b200 import binding
+    d = binding.TensorDesc(bits=4, rows=4, cols=64)
+    h = binding.HParams(sigma=0.5, lr=1.0, gamma=0.9, n_pop=4)
+    w = torch.zeros(128, dtype=torch.uint8)
+    with pytest.raises(binding.QesError):
+        binding.qes_perturb(d, w, w, None, 1, h, stream=0)

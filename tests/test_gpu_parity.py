@@ -1,0 +1,245 @@
+"""Parity of the CUDA library (through its C ABI) against the CPU oracle, element by element.
+
+Rules (the benchmark spec): packed codes bit-exact, except elements whose pre-rounding value u lies within
+1e-5 of a rounding boundary in any generation (counted, reported, never silently skipped);
+residuals within 1e-5 absolute on the remaining elements.  qes_perturb has no such band: exact.
+"""
+import numpy as np
+import pytest
+
+from paper_2602_03120_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+BAND = 1e-5
+TOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def qes():
+    import torch
+    from paper_2602_03120_b200 import binding
+    assert torch.cuda.is_available()
+    binding.load()
+    return binding
+
+
+def _dev(a):
+    import torch
+    a = np.ascontiguousarray(a)
+    if a.dtype == np.uint64:
+        a = a.view(np.int64)
+    return torch.from_numpy(a).cuda()
+
+
+def _host(t):
+    return t.cpu().numpy()
+
+
+def _case(qo, qes, bits, rows, cols, group=0, off=0, qmin=None, qmax=None, seed=0):
+    n = rows * cols
+    rng = np.random.default_rng([seed, rows, cols])
+    packed = rng.integers(0, 256, size=n if bits == 8 else n // 2, dtype=np.uint8)
+    if qmin is not None:   # keep codes inside a narrower range
+        codes = np.clip(qo.unpack(bits, packed, n), qmin, qmax)
+        packed = qo.pack(bits, codes)
+    to = qo.Tensor(bits=bits, rows=rows, cols=cols, group_size=group, elem_offset=off, qmin=qmin, qmax=qmax)
+    tg = qes.TensorDesc(bits=bits, rows=rows, cols=cols, group_size=group, elem_offset=off, qmin=qmin, qmax=qmax)
+    n_scales = rows * (cols // group) if group else rows
+    scales = rng.lognormal(-4.0, 0.3, size=n_scales).astype(np.float16)
+    return to, tg, packed, scales
+
+
+def _hp(qo, qes, **kw):
+    return qo.HParams(**kw), qes.HParams(**kw)
+
+
+def _compare_update(qo, packed_gpu, bits, ref, what=""):
+    got = qo.unpack(bits, packed_gpu, ref["w_new"].size)
+    near = ref["band"] < BAND
+    bad = (got != ref["w_new"]) & ~near
+    assert not bad.any(), f"{what}: {bad.sum()} codes differ outside the rounding band (near-band: {near.sum()})"
+    # inside the band either rounding is acceptable, but it must be one of the two neighbours
+    assert np.all(np.abs(got[near] - ref["w_new"][near]) <= 1)
+    return int(near.sum())
+
+
+@pytest.mark.parametrize("bits,rows,cols,off", [(4, 37, 352, 0), (8, 21, 160, 96), (4, 1, 32, 0),
+                                                (4, 9, 4096, (1 << 34) + 64), (8, 3, 64, (1 << 40))])
+def test_perturb_bit_exact(qo, qes, bits, rows, cols, off):
+    to, tg, packed, _ = _case(qo, qes, bits, rows, cols, off=off)
+    for mode in (0, 1):
+        for sigma in (0.5, 2.0):          # 2.0 compiles in the 4-bit limit on delta
+            ho, hg = _hp(qo, qes, sigma=sigma, lr=1.0, gamma=0.9, n_pop=1, boundary_mode=mode)
+            seed = 0xC0FFEE_0000_0000 + rows
+            w_in = _dev(packed); w_out = _dev(np.zeros_like(packed))
+            qes.qes_perturb(tg, w_in, w_out, None, seed, hg)
+            ref = qo.perturb(to, packed, None, seed, ho)
+            assert np.array_equal(_host(w_out), qo.pack(bits, ref))
+            assert np.array_equal(_host(w_in), packed)
+            qes.qes_perturb(tg, w_in, w_in, None, seed, hg)     # exact aliasing is allowed
+            assert np.array_equal(_host(w_in), qo.pack(bits, ref))
+    assert np.any(ref != qo.unpack(bits, packed, rows * cols))
+
+
+@pytest.mark.parametrize("bits,rows,cols,group,N,K,mode", [
+    (4, 67, 1024, 128, 8, 4, 0), (4, 5, 96, 32, 3, 0, 0), (8, 33, 544, 0, 5, 3, 0),
+    (4, 19, 640, 64, 7, 6, 1), (8, 1, 32, 0, 1, 1, 1)])
+def test_stateless_update_and_replay(qo, qes, bits, rows, cols, group, N, K, mode):
+    import torch
+    to, tg, packed, scales = _case(qo, qes, bits, rows, cols, group=group, off=32 * 1001)
+    ho, hg = _hp(qo, qes, sigma=0.5, lr=1.0, gamma=0.9, n_pop=N, boundary_mode=mode)
+    seeds, fit = wl.draw_seeds(K + 1, N, stream=rows), wl.draw_fitness(K + 1, N, stream=rows)
+    w = _dev(packed); stats = torch.zeros(4, dtype=torch.int64, device="cuda")
+    qes.qes_update(tg, w, None, _dev(seeds), _dev(fit), K, None, hg, stats=stats)
+    ref = qo.update(to, packed, None, seeds, fit, K, ho)
+    n_near = _compare_update(qo, _host(w), bits, ref, "stateless update")
+    st = _host(stats)
+    far = ref["band"] >= BAND
+    changed = (ref["w_new"] != qo.unpack(bits, packed, rows * cols))
+    assert abs(int(st[0]) - int(changed.sum())) <= n_near
+    assert abs(int(st[1]) - int(ref["gate_final"].sum())) <= n_near
+    assert abs(int(st[2]) - int(ref["gate_replay"].sum())) <= n_near * max(K, 1)
+    assert abs(int(st[3]) - int(ref["attempted"].sum())) <= n_near
+    # history loop alone
+    res = torch.full((rows * cols,), 7.0, dtype=torch.float32, device="cuda")
+    qes.qes_replay_residual(tg, _dev(packed), None, _dev(seeds[:K]), _dev(fit[:K]), K, hg, res)
+    rr = qo.replay_residual(to, packed, None, seeds[:K], fit[:K], K, ho)
+    farr = rr["band"] >= BAND
+    assert np.abs(_host(res).astype(np.float64) - rr["e"])[farr].max(initial=0.0) <= TOL
+    assert farr.mean() > 0.99
+
+
+def test_stored_residual_step(qo, qes):
+    import torch
+    to, tg, packed, _ = _case(qo, qes, 4, 41, 288)
+    ho, hg = _hp(qo, qes, sigma=0.5, lr=1.0, gamma=0.9, n_pop=8)
+    n = 41 * 288
+    e_in = np.random.default_rng(0).uniform(-0.5, 0.5, n).astype(np.float32)
+    seeds, fit = wl.draw_seeds(1, 8, stream=77), wl.draw_fitness(1, 8, stream=77)
+    w = _dev(packed); e = _dev(e_in)
+    qes.qes_update(tg, w, None, _dev(seeds), _dev(fit), 0, e, hg)
+    ref = qo.update(to, packed, None, seeds, fit, 0, ho, residual_in=e_in)
+    _compare_update(qo, _host(w), 4, ref, "stored residual")
+    far = ref["band"] >= BAND
+    assert np.abs(_host(e).astype(np.float64) - ref["e_new"])[far].max() <= TOL
+
+
+def test_weight_unit_sigma_reads_group_scales(qo, qes):
+    for bits, rows, cols, group in ((4, 23, 512, 128), (4, 7, 256, 64), (8, 29, 96, 0)):
+        to, tg, packed, scales = _case(qo, qes, bits, rows, cols, group=group)
+        kw = dict(sigma=0.012, lr=1.0, gamma=0.9, n_pop=6, sigma_unit=1)
+        ho, hg = _hp(qo, qes, **kw)
+        seeds, fit = wl.draw_seeds(3, 6, stream=5), wl.draw_fitness(3, 6, stream=5)
+        w = _dev(packed)
+        qes.qes_update(tg, w, _dev(scales), _dev(seeds), _dev(fit), 2, None, hg)
+        ref = qo.update(to, packed, scales, seeds, fit, 2, ho)
+        _compare_update(qo, _host(w), bits, ref, "weight-unit sigma")
+        wp = _dev(np.zeros_like(packed))
+        qes.qes_perturb(tg, _dev(packed), wp, _dev(scales), 99, hg)
+        assert np.array_equal(_host(wp), qo.pack(bits, qo.perturb(to, packed, scales, 99, ho)))
+
+
+def test_symmetric_grid_range(qo, qes):
+    """App. A grid: codes in [-(2^(B-1)-1), 2^(B-1)-1]."""
+    to, tg, packed, _ = _case(qo, qes, 4, 16, 256, qmin=-7, qmax=7)
+    ho, hg = _hp(qo, qes, sigma=0.5, lr=1.0, gamma=0.9, n_pop=8)
+    seeds, fit = wl.draw_seeds(3, 8, stream=6), wl.draw_fitness(3, 8, stream=6)
+    w = _dev(packed)
+    qes.qes_update(tg, w, None, _dev(seeds), _dev(fit), 2, None, hg)
+    ref = qo.update(to, packed, None, seeds, fit, 2, ho)
+    _compare_update(qo, _host(w), 4, ref, "symmetric grid")
+    got = qo.unpack(4, _host(w), 16 * 256)
+    assert got.min() >= -7 and got.max() <= 7
+
+
+def test_split_invariance_and_determinism(qo, qes):
+    to, tg, packed, _ = _case(qo, qes, 4, 64, 256, off=1 << 21)
+    _, hg = _hp(qo, qes, sigma=0.5, lr=1.0, gamma=0.9, n_pop=8)
+    seeds, fit = _dev(wl.draw_seeds(4, 8)), _dev(wl.draw_fitness(4, 8))
+    whole = _dev(packed)
+    qes.qes_update(tg, whole, None, seeds, fit, 3, None, hg)
+    again = _dev(packed)
+    qes.qes_update(tg, again, None, seeds, fit, 3, None, hg)
+    assert np.array_equal(_host(whole), _host(again))
+    half = 32 * 256
+    top = qes.TensorDesc(bits=4, rows=32, cols=256, elem_offset=1 << 21)
+    bot = qes.TensorDesc(bits=4, rows=32, cols=256, elem_offset=(1 << 21) + half)
+    a, b = _dev(packed[:half // 2]), _dev(packed[half // 2:])
+    qes.qes_update(top, a, None, seeds, fit, 3, None, hg)
+    qes.qes_update(bot, b, None, seeds, fit, 3, None, hg)
+    assert np.array_equal(np.concatenate([_host(a), _host(b)]), _host(whole))
+
+
+def test_empty_history_and_zero_fitness(qo, qes):
+    import torch
+    to, tg, packed, _ = _case(qo, qes, 4, 4, 128)
+    _, hg = _hp(qo, qes, sigma=0.5, lr=1.0, gamma=0.9, n_pop=4)
+    res = torch.full((512,), 3.0, dtype=torch.float32, device="cuda")
+    qes.qes_replay_residual(tg, _dev(packed), None, None, None, 0, hg, res)
+    assert np.all(_host(res) == 0.0)
+    w = _dev(packed)
+    qes.qes_update(tg, w, None, _dev(wl.draw_seeds(3, 4)), _dev(np.zeros((3, 4), np.float32)), 2, None, hg)
+    assert np.array_equal(_host(w), packed)
+
+
+def test_config1_full_matrix(qo, qes):
+    """Benchmark configuration 1 in full: 4096x4096 INT4, N = 8, K = 4, every element compared."""
+    cfg = wl.WORKLOADS["matrix4096_int4"]
+    t = cfg.tensors[0]
+    packed = wl.draw_codes(cfg, 0)
+    seeds, fit = wl.draw_seeds(cfg.K + 1, cfg.n_pop), wl.draw_fitness(cfg.K + 1, cfg.n_pop, cfg.reward_dist)
+    kw = dict(sigma=cfg.sigma, lr=cfg.lr, gamma=cfg.gamma, n_pop=cfg.n_pop)
+    ho, hg = _hp(qo, qes, **kw)
+    to = qo.Tensor(bits=4, rows=t.rows, cols=t.cols, group_size=cfg.group_size)
+    tg = qes.TensorDesc(bits=4, rows=t.rows, cols=t.cols, group_size=cfg.group_size)
+    w = _dev(packed)
+    qes.qes_update(tg, w, None, _dev(seeds), _dev(fit), cfg.K, None, hg)
+    ref = qo.update(to, packed, None, seeds, fit, cfg.K, ho)
+    n_near = _compare_update(qo, _host(w), 4, ref, "config 1")
+    print(f"config 1: {t.numel} elements, {n_near} inside the 1e-5 rounding band")
+    assert n_near < 1e-3 * t.numel
+    assert (ref["w_new"] != qo.unpack(4, packed, t.numel)).mean() > 0.01
+
+
+@pytest.mark.parametrize("name", ["decoder7b_int4", "decoder7b_int8", "decoder8b_int4"])
+def test_full_size_tensors_sampled(qo, qes, name):
+    """Full-size tensors of the large configurations in the benchmark's launch configuration (one call per
+    tensor, the configuration's N and K), oracle on sampled 32-element words incl. first and last."""
+    cfg = wl.WORKLOADS[name]
+    kw = dict(sigma=cfg.sigma, lr=cfg.lr, gamma=cfg.gamma, n_pop=cfg.n_pop)
+    ho, hg = _hp(qo, qes, **kw)
+    seeds, fit = wl.draw_seeds(cfg.K + 1, cfg.n_pop), wl.draw_fitness(cfg.K + 1, cfg.n_pop, cfg.reward_dist)
+    ds, df = _dev(seeds), _dev(fit)
+    per_tensor = 2048 if cfg.K <= 16 else 256
+    picks = [1, 6, len(cfg.tensors) - 1] if cfg.K <= 16 else [len(cfg.tensors) - 6]   # k_proj, down_proj, last / one k_proj
+    total_near = 0
+    for ti in picks:
+        t = cfg.tensors[ti]
+        packed = wl.draw_codes(cfg, ti)
+        to = qo.Tensor(bits=cfg.bits, rows=t.rows, cols=t.cols, group_size=cfg.group_size, elem_offset=t.elem_offset)
+        tg = qes.TensorDesc(bits=cfg.bits, rows=t.rows, cols=t.cols, group_size=cfg.group_size, elem_offset=t.elem_offset)
+        w = _dev(packed)
+        qes.qes_update(tg, w, None, ds, df, cfg.K, None, hg)
+        idx = wl.sample_elements(t.numel, per_tensor, stream=ti)
+        ref = qo.update(to, packed, None, seeds, fit, cfg.K, ho, idx=idx)
+        got = qo.unpack(cfg.bits, _host(w), t.numel)[idx]
+        near = ref["band"] < BAND
+        assert not np.any((got != ref["w_new"]) & ~near), f"{name} tensor {ti}"
+        total_near += int(near.sum())
+        # properties that hold at any size: range, and untouched where the oracle sample is untouched
+        assert got.min() >= cfg.qmin and got.max() <= cfg.qmax
+    print(f"{name}: near-band sampled elements {total_near}")
+
+
+def test_perturb_delta_is_the_delta_the_update_sums(qo, qes):
+    to, tg, packed, _ = _case(qo, qes, 8, 8, 128)
+    packed = np.zeros_like(packed)           # far from the boundary: perturb output is delta itself
+    ho, hg = _hp(qo, qes, sigma=1.0, lr=1.0, gamma=0.0, n_pop=1)
+    seed = 424242
+    wp = _dev(np.zeros_like(packed))
+    qes.qes_perturb(tg, _dev(packed), wp, None, seed, hg)
+    w = _dev(packed)
+    qes.qes_update(tg, w, None, _dev(np.array([[seed]], np.uint64)), _dev(np.array([[1.0]], np.float32)), 0, None, hg)
+    assert np.array_equal(_host(wp), _host(w))
+    assert np.array_equal(qo.unpack(8, _host(wp), 1024), qo.delta(seed, np.arange(1024, dtype=np.uint64), 1.0)[0])
