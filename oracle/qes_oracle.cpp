@@ -15,7 +15,8 @@
 // Two tiers:
 //   tier 0 ("plain"): Gaussian in double with libm log/sqrt/sin/cos.
 //   tier 1 ("spec") : Gaussian by a fixed sequence of IEEE fp32 operations
-//                     ("BM24") that a GPU can reproduce bit for bit.
+//                     ("BM24") that a GPU can reproduce bit for bit; the rounding
+//                     decision of Eq. 3 on that fp32 value is taken exactly.
 // Everything after the noise sample (sum, u, round, gate, residual) is double.
 //
 // Build: g++ -O2 -std=c++17 -ffp-contract=off -fPIC -shared -pthread
@@ -100,12 +101,16 @@ void bm24_cossin(uint32_t r1, float* c_out, float* s_out) {
     }
 }
 
-// Eq. 3 in fp32: delta = floor(x) + [v < x - floor(x)], then the 4-bit range of
-// the perturbation tensor (App. A "4-bit stochastically rounded perturbation").
+// Eq. 3: delta = floor(x) + b, b ~ Bernoulli(x - floor(x)), realised as b = [v < x - floor(x)]
+// with the 24-bit uniform v = (word >> 8) / 2^24.  x is the fp32 value sigma_eff * eps; its
+// fractional part and the comparison are evaluated exactly (both are exact in double), so
+// P(b = 1) is the fractional part of x to within the 2^-24 grid of v and nothing else.  Then the
+// 4-bit range of the perturbation tensor (App. A "4-bit stochastically rounded perturbation").
 int stochastic_round_f32(float x, uint32_t rword) {
-    float fl = std::floor(x);
-    float frac = x - fl;
-    float v = (float)(rword >> 8) * 0x1p-24f;  // exact, [0,1)
+    double xd = (double)x;
+    double fl = std::floor(xd);
+    double frac = xd - fl;                          // exact
+    double v = (double)(rword >> 8) / 16777216.0;   // exact, [0,1)
     int d = (int)fl + (v < frac ? 1 : 0);
     return std::min(7, std::max(-8, d));
 }

@@ -1,6 +1,7 @@
 """Pins for the oracle's noise generator: Philox known answers, Box-Muller against libm,
 stochastic rounding (Eq. 3) against its definition and its expectation."""
 import os
+from fractions import Fraction
 
 import numpy as np
 from scipy import stats
@@ -80,9 +81,10 @@ def test_delta_wiring_matches_manual_composition(qo):
         trig = s[0] if (int(j) & 1) else c[0]
         xx = np.float32(np.float32(sig) * R[0]) * trig
         assert np.float32(xx) == np.float32(x[i])
-        v = np.float32(int(r[3 if (int(j) & 1) else 2]) >> 8) * np.float32(2.0 ** -24)
-        fl = np.floor(np.float32(xx))
-        want = int(fl) + (1 if v < np.float32(np.float32(xx) - fl) else 0)
+        # Eq. 3 decided exactly: 24-bit integer uniform against the exact fractional part of the fp32 x
+        xq = Fraction(float(np.float32(xx)))
+        fl = xq.numerator // xq.denominator
+        want = fl + (1 if Fraction(int(r[3 if (int(j) & 1) else 2]) >> 8, 1 << 24) < xq - fl else 0)
         assert d[i] == max(-8, min(7, want))
 
 
@@ -110,6 +112,21 @@ def test_stochastic_rounding_unbiased_and_two_valued(qo):
             assert np.all(d == fl)
     # 4-bit range of the perturbation tensor
     assert qo.stochastic_round(9.5, 0) == 7 and qo.stochastic_round(-11.2, 0xffffffff) == -8
+
+
+def test_bernoulli_threshold_is_the_exact_fraction(qo):
+    """Eq. 3: b ~ Bernoulli(x - floor(x)).  For x in (-1/2, 0) the difference x - floor(x) does not fit
+    fp32; the decision must use its exact value, so of the 2^24 equally likely uniforms exactly
+    ceil((x - floor(x)) * 2^24) give b = 1."""
+    x = -(2.0 ** -3 + 3 * 2.0 ** -26)                 # exact in fp32; (x + 1) * 2^24 = 14680063.25
+    assert float(np.float32(x)) == x
+    assert qo.stochastic_round(x, 14680063 << 8) == 0     # v = 14680063 / 2^24 < x + 1  -> b = 1
+    assert qo.stochastic_round(x, 14680064 << 8) == -1    # v = 14680064 / 2^24 > x + 1  -> b = 0
+    assert qo.stochastic_round(x, (14680063 << 8) | 0xff) == 0   # the low 8 bits of the word are unused
+    # integer x: fraction 0, b = 0 for every uniform, including v = 0
+    assert qo.stochastic_round(2.0, 0) == 2 and qo.stochastic_round(-3.0, 0) == -3
+    # smallest positive fraction: only v = 0 gives b = 1
+    assert qo.stochastic_round(2.0 ** -30, 0) == 1 and qo.stochastic_round(2.0 ** -30, 1 << 8) == 0
 
 
 def test_expected_delta_equals_sigma_eps(qo):
