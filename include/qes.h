@@ -23,6 +23,8 @@
  *    Philox4x32-10(key = seed, counter = J >> 1) -> Box-Muller -> sigma scaling -> stochastic
  *    rounding (Eq. 3), limited to the 4-bit range [-8, 7] (App. A).  Results depend only on
  *    (seed, J): any split of a model into tensors, any grid size, gives the same bits.
+ *    With sigma_unit == QES_SIGMA_WEIGHT, sigma / scale above 2^40 is treated as 2^40 (every
+ *    non-zero sample saturates the 4-bit range long before).
  *  - Fitness values are the already normalised rewards F_i (Algorithm 1, "Normalize reward").
  *  - Return value: QES_OK, or a negative qes_status; on any error nothing was launched and no
  *    buffer was touched.
@@ -45,7 +47,7 @@ typedef enum {
     QES_ERR_BAD_HPARAM = -5,  /* sigma <= 0, n_pop <= 0, K < 0, gamma outside [0,1], qmin >= qmax, range outside the code width */
     QES_ERR_BAD_MODE = -6,    /* unknown sigma_unit / boundary_mode, or residual_inout given with K > 0 */
     QES_ERR_CUDA = -7,        /* the launch reported a CUDA error (cudaGetLastError) */
-    QES_ERR_TOO_LARGE = -8    /* the (K+1)*n_pop table does not fit the kernel's shared-memory staging */
+    QES_ERR_TOO_LARGE = -8    /* n_pop exceeds what one generation's shared-memory staging holds (1066 members) */
 } qes_status;
 
 enum { QES_SIGMA_GRID = 0, QES_SIGMA_WEIGHT = 1 };   /* unit of hparams.sigma: grid steps | weight units (sigma_g = sigma / scale_g) */
@@ -104,15 +106,29 @@ int qes_update(const qes_tensor_desc* desc, void* w_inout, const void* scales_f1
                const qes_hparams* hparams, uint64_t* stats, void* cuda_stream);
 
 /*
+ * The Box-Muller factors of the noise contract on their own (Sec. 3.2 "RNG(seed)"; the paper
+ * names no generator, this library fixes one): for each i, radius[i] = sqrt(-2 ln u1) with
+ * u1 = ((r0[i] >> 8) + 1) / 2^24, and (cosine[i], sine[i]) of 2*pi*u2 with u2 = (r1[i] >> 8) / 2^24,
+ * each by the library's fixed fp32 operation sequence.  Lets a caller check that sequence on its
+ * whole domain (2^24 values per factor).  All five arrays are DEVICE pointers to n elements,
+ * owned by the caller; n == 0 is a no-op.  Enqueues on cuda_stream, does not synchronise.
+ */
+int qes_gaussian_factors(const uint32_t* r0, const uint32_t* r1, int64_t n, float* radius, float* cosine,
+                         float* sine, void* cuda_stream);
+
+/*
  * Arithmetic-pipe throughput probes used to derive the ALU roofline (no counterpart in the
  * paper).  Runs `iters` dependent-chain iterations of one instruction kind on every lane of a
  * full grid and writes the elapsed device time in milliseconds to *ms_out (HOST pointer) and
  * the number of lane-operations performed to *ops_out (HOST pointer).  sink_dev is a DEVICE
  * buffer of at least 4 bytes owned by the caller (the probes keep their results live by a store
  * that is practically never taken).  Runs on the default stream and synchronises.
- *   kind: 0 mul.wide.u32  1 lop3 (xor3)  2 fma.rn.f32  3 mul.hi.u32  4 cvt.rn.f32.u32
+ *   kind: 0 mul.wide.u32 (low half kept)  1 lop3 (xor3)  2 fma.rn.f32  3 mul.hi.u32  4 cvt.rn.f32.u32
  *         5 sqrt.rn.f32   6 cvt.rmi (floor)  7 mad.lo.u32  8 Philox round (2 wide multiplies + 2 xor3)
- *         9 rsqrt.approx.f32 (special-function unit)
+ *         9 rsqrt.approx.f32 (special-function unit)  10-17 add, shift, fp32 add/mul/compare/min, cvt.rzi
+ *         18 mad.wide.u32 with the 64-bit result live  19 mul.wide.u32 + xor3 of both halves (counted
+ *         per step)  20/21/22 the same plus 1/2/4 independent fp32 fma per step
+ *         100-109 two-kind mixes (see the binding's PROBE_KINDS)
  */
 int qes_pipe_probe(int32_t kind, int32_t iters, void* sink_dev, float* ms_out, double* ops_out);
 

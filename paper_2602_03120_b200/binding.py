@@ -88,6 +88,8 @@ def load() -> C.CDLL:
         lib.qes_replay_residual.argtypes = [C.POINTER(_TensorDesc), vp, vp, vp, vp, i32, C.POINTER(_HParams), vp, vp]
         lib.qes_update.restype = C.c_int
         lib.qes_update.argtypes = [C.POINTER(_TensorDesc), vp, vp, vp, vp, i32, vp, C.POINTER(_HParams), vp, vp]
+        lib.qes_gaussian_factors.restype = C.c_int
+        lib.qes_gaussian_factors.argtypes = [vp, vp, C.c_int64, vp, vp, vp, vp]
         lib.qes_pipe_probe.restype = C.c_int
         lib.qes_pipe_probe.argtypes = [i32, i32, vp, C.POINTER(C.c_float), C.POINTER(C.c_double)]
         lib.qes_strerror.restype = C.c_char_p
@@ -170,10 +172,23 @@ def qes_update(desc: TensorDesc, w_inout, scales_f16, seeds, fitness, K: int, re
     _check(rc)
 
 
+def qes_gaussian_factors(r0, r1, radius, cosine, sine, stream=None) -> None:
+    """Box-Muller factors of the noise contract for 32-bit word pairs (uint32/int32 in, float32 out)."""
+    n = r0.numel()
+    words = (torch.int32, torch.uint32)
+    rc = load().qes_gaussian_factors(_ptr(r0, dtype=words, nbytes=4 * n, name="r0"), _ptr(r1, dtype=words, nbytes=4 * n, name="r1"),
+                                     n, _ptr(radius, dtype=torch.float32, nbytes=4 * n, name="radius"),
+                                     _ptr(cosine, dtype=torch.float32, nbytes=4 * n, name="cosine"),
+                                     _ptr(sine, dtype=torch.float32, nbytes=4 * n, name="sine"), _stream(stream))
+    _check(rc)
+
+
 PROBE_KINDS = {0: "mul.wide.u32", 1: "lop3.xor3", 2: "fma.rn.f32", 3: "mul.hi.u32", 4: "cvt.rn.f32.u32",
                5: "sqrt.rn.f32", 6: "cvt.rmi.f32.f32", 7: "mad.lo.u32", 8: "philox round (2 mul.wide + 2 xor3)",
                9: "rsqrt.approx.f32", 10: "add.u32", 11: "shr.u32", 12: "add.rn.f32", 13: "mul.rn.f32",
-               14: "setp.lt.f32 + selp", 15: "min.f32", 16: "cvt.rzi.s32.f32", 17: "set.lt.f32 (1.0/0.0)",
+               14: "setp.lt.f32 + selp", 15: "min.f32", 16: "cvt.rzi.s32.f32", 17: "set.lt.f32 (1.0/0.0)", 18: "mad.wide.u32 (64-bit result live)",
+               19: "mul.wide.u32 + xor3 of both halves (steps)", 20: "mul.wide + xor3 + 1 fma (steps)",
+               21: "mul.wide + xor3 + 2 fma (steps)", 22: "mul.wide + xor3 + 4 fma (steps)",
                100: "mix mul.wide + xor3", 101: "mix fma + xor3", 102: "mix mul.wide + fma", 103: "mix cvt.f32.u32 + xor3",
                104: "mix cvt.f32.u32 + mul.wide", 105: "mix floor + rsqrt", 106: "mix floor + fma", 107: "mix add + xor3",
                108: "mix fadd + mul.wide", 109: "mix setp/selp + fma"}

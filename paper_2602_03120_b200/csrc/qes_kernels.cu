@@ -1,23 +1,40 @@
 // Kernels and C ABI of the QES parameter pass (sm_100a).  See include/qes.h for the contract.
 //
-// Work decomposition: one thread owns 16 consecutive codes (8 Philox pairs): a 64-bit load for
-// INT4, a 128-bit load for INT8, so a warp reads and writes whole 256 B / 512 B segments.  The
-// (generation, member) table of seeds and fitness values is staged once per CTA in shared
-// memory; every thread then walks it in the same order, so each table read is a broadcast.
-// Per member the ten Philox round keys are expanded once per thread and reused by its 8 pairs.
-// The path is bound by integer/fp32 issue slots, not by HBM: a code costs 1 byte of traffic
-// but N*(K+1) noise samples of ~50 arithmetic operations each.
+// Work decomposition: one thread owns 2*kPairs consecutive codes (kPairs Philox calls per seed):
+// with kPairs = 8 a 64-bit load for INT4 and a 128-bit load for INT8, so a warp reads and writes
+// whole 256 B / 512 B segments, once.  Everything else is arithmetic in registers: a code costs
+// one byte of HBM traffic but N*(K+1) noise samples of ~50 operations each, so the kernels are
+// bound by instruction issue and by the integer / wide-multiply pipes, never by memory.
+//
+// Per generation the CTA stages, in shared memory, the ten Philox round keys of each of the N
+// seeds next to the member's fitness (96 B per member, double-buffered so one barrier per
+// generation suffices); every thread then walks the members in the same order, each table read
+// is a broadcast, and a seed's keys are fetched with five 128-bit loads instead of being
+// re-derived by 18 additions per thread.  The residual e and the weighted sums S of Eqs. 5-8
+// never leave registers between generations (Algorithm 2 keeps no O(d) state).
 #include "qes_device.cuh"
 #include "../../include/qes.h"
+
+#ifndef QES_PAIRS
+#define QES_PAIRS 4
+#endif
+#ifndef QES_MIN_BLOCKS
+#define QES_MIN_BLOCKS 2
+#endif
 
 namespace qes {
 
 enum PassMode : int { kStateless = 0, kStoredResidual = 1, kReplayOnly = 2 };
 
+constexpr int kThreads = 256;
+constexpr int kPairs = QES_PAIRS;
+constexpr int kCodesPerThread = 2 * kPairs;
+constexpr int kSeedStride = 24;   // 32-bit words per staged member: a[10], b[10], fitness, 3 pad
+
 struct PassParams {
     const void* w_in;
     void* w_out;
-    const __half_raw* scales;   // nullable
+    const unsigned short* scales;   // nullable, IEEE binary16 bits
     const uint64_t* seeds;
     const float* fitness;
     float* residual;            // stored-residual in/out, or replay output
@@ -33,6 +50,7 @@ struct PassParams {
     int32_t weight_unit;
     float sigma, coef, gamma;   // coef = lr / (n_pop * sigma)
     float qmin, qmax;
+    int32_t qmin_i, qmax_i;
 };
 
 __device__ __forceinline__ float half_bits_to_float(unsigned short h) {
@@ -40,13 +58,15 @@ __device__ __forceinline__ float half_bits_to_float(unsigned short h) {
     return __half2float(__half(r));
 }
 
-__device__ __forceinline__ float chunk_sigma(const PassParams& p, int64_t chunk) {
-    if (!p.weight_unit) return p.sigma;
+// -sigma_eff * 2^24 for the codes of one thread, sigma_eff = sigma in grid steps (they share a
+// scale: groups span >= 32 codes).  sigma / scale is capped at 2^40: beyond that every non-zero
+// sample already saturates the 4-bit range of delta, so the cap changes nothing.
+__device__ __forceinline__ float chunk_neg_sigma24(const PassParams& p, int64_t chunk) {
+    if (!p.weight_unit) return -p.sigma * 0x1p24f;
     int64_t j = chunk * kCodesPerThread;
     int64_t row = j / p.cols;
     int64_t g = p.group_size > 0 ? row * (p.cols / p.group_size) + (j - row * p.cols) / p.group_size : row;
-    unsigned short h = reinterpret_cast<const unsigned short*>(p.scales)[g];
-    return __fdiv_rn(p.sigma, half_bits_to_float(h));
+    return -fminf(__fdiv_rn(p.sigma, half_bits_to_float(p.scales[g])), 0x1p40f) * 0x1p24f;
 }
 
 // Eq. 4 (gate) or saturation: the step actually applied to code w for a rounded step.
@@ -56,125 +76,215 @@ __device__ __forceinline__ float applied_step(float w, float step, float qmin, f
     return fminf(fmaxf(target, qmin), qmax) - w;
 }
 
+// The same rule on integer codes: the code after the step.
+__device__ __forceinline__ int applied_code(int w, int step, int qmin, int qmax, int boundary_mode) {
+    int target = w + step;
+    if (boundary_mode == QES_BOUNDARY_GATE) return (target >= qmin && target <= qmax) ? target : w;
+    return min(max(target, qmin), qmax);
+}
+
+// Algorithm 1, member loop: W' = Gate(W + delta_i).  The member's round keys are computed on the
+// host and arrive as kernel parameters, i.e. as constant-bank operands.
 template <int BITS, bool CLAMP_DELTA>
-__global__ void __launch_bounds__(256) perturb_kernel(PassParams p, uint32_t key0, uint32_t key1) {
+__global__ void __launch_bounds__(kThreads) perturb_kernel(PassParams p, RoundKeys rk) {
     int64_t chunk = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (chunk >= p.n_chunks) return;
-    Chunk<BITS> w;
+    Chunk<BITS, kPairs> w;
     w.load(p.w_in, chunk);
-    float sig = chunk_sigma(p, chunk);
-    uint64_t pair0 = (p.elem_offset + (uint64_t)chunk * kCodesPerThread) >> 1;
-    uint32_t c0 = (uint32_t)pair0, c1 = (uint32_t)(pair0 >> 32);
-    RoundKeys rk = make_round_keys(key0, key1);
-    Chunk<BITS> out;
+    float nsig24 = chunk_neg_sigma24(p, chunk);
+    uint64_t pair0 = (p.elem_offset >> 1) + (uint64_t)chunk * kPairs;
+    uint32_t x0 = (uint32_t)pair0, y = (uint32_t)(pair0 >> 32);
+    SeedConst sc = make_seed_const(y, rk);
+    Chunk<BITS, kPairs> out;
     out.clear();
 #pragma unroll
-    for (int i = 0; i < kCodesPerThread / 2; ++i) {
-        float d0, d1;
-        delta_pair<CLAMP_DELTA>(c0 + i, c1, rk, sig, d0, d1);
+    for (int i = 0; i < kPairs; ++i) {
+        uint32_t r0, r1, r2, r3;
+        philox_tail(make_pair_const(x0 + i), sc, rk, r0, r1, r2, r3);
+        int z0, z1;
+        pair_rounding_sums<CLAMP_DELTA>(r0, r1, r2, r3, nsig24, z0, z1);
         int w0 = w.get(2 * i), w1 = w.get(2 * i + 1);
-        out.put(2 * i, w0 + (int)applied_step((float)w0, d0, p.qmin, p.qmax, p.boundary_mode));
-        out.put(2 * i + 1, w1 + (int)applied_step((float)w1, d1, p.qmin, p.qmax, p.boundary_mode));
+        out.put(2 * i, applied_code(w0, -neg_delta<CLAMP_DELTA>(z0), p.qmin_i, p.qmax_i, p.boundary_mode));
+        out.put(2 * i + 1, applied_code(w1, -neg_delta<CLAMP_DELTA>(z1), p.qmin_i, p.qmax_i, p.boundary_mode));
     }
     out.store(p.w_out, chunk);
 }
 
+// Expands the seeds of one generation into round keys, next to the fitness values (stored as
+// -F * 2^-24, the factor that turns the kernel's -delta * 2^24 back into F * delta).
+__device__ __forceinline__ void stage_generation(uint32_t* buf, const uint64_t* seeds, const float* fitness, int n_pop) {
+    for (int i = threadIdx.x; i < n_pop; i += kThreads) {
+        uint64_t s = seeds[i];
+        RoundKeys rk = make_round_keys((uint32_t)s, (uint32_t)(s >> 32));
+        uint4* d = reinterpret_cast<uint4*>(buf + i * kSeedStride);
+        d[0] = make_uint4(rk.a[0], rk.a[1], rk.a[2], rk.a[3]);
+        d[1] = make_uint4(rk.a[4], rk.a[5], rk.a[6], rk.a[7]);
+        d[2] = make_uint4(rk.a[8], rk.a[9], rk.b[0], rk.b[1]);
+        d[3] = make_uint4(rk.b[2], rk.b[3], rk.b[4], rk.b[5]);
+        d[4] = make_uint4(rk.b[6], rk.b[7], rk.b[8], rk.b[9]);
+        d[5] = make_uint4(__float_as_uint(fitness[i] * -0x1p-24f), 0u, 0u, 0u);   // pairs with -delta * 2^24
+    }
+}
+
+__device__ __forceinline__ RoundKeys load_round_keys(const uint32_t* entry, float& fit) {
+    const uint4* q = reinterpret_cast<const uint4*>(entry);
+    uint4 k0 = q[0], k1 = q[1], k2 = q[2], k3 = q[3], k4 = q[4];
+    fit = __uint_as_float(entry[20]);
+    RoundKeys rk;
+    rk.a[0] = k0.x; rk.a[1] = k0.y; rk.a[2] = k0.z; rk.a[3] = k0.w;
+    rk.a[4] = k1.x; rk.a[5] = k1.y; rk.a[6] = k1.z; rk.a[7] = k1.w;
+    rk.a[8] = k2.x; rk.a[9] = k2.y; rk.b[0] = k2.z; rk.b[1] = k2.w;
+    rk.b[2] = k3.x; rk.b[3] = k3.y; rk.b[4] = k3.z; rk.b[5] = k3.w;
+    rk.b[6] = k4.x; rk.b[7] = k4.y; rk.b[8] = k4.z; rk.b[9] = k4.w;
+    return rk;
+}
+
 // Algorithm 2 (stateless), Algorithm 1's update lines (stored residual) or the history loop
-// alone (replay only), selected by p.mode.  Shared memory: generations*n_pop (seed, fitness).
-template <int BITS, bool CLAMP_DELTA>
-__global__ void __launch_bounds__(256) pass_kernel(PassParams p) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    const int entries = p.generations * p.n_pop;
-    uint2* s_key = reinterpret_cast<uint2*>(smem_raw);
-    float* s_fit = reinterpret_cast<float*>(smem_raw + (size_t)entries * sizeof(uint2));
-    for (int i = threadIdx.x; i < entries; i += blockDim.x) {
-        uint64_t s = p.seeds[i];
-        s_key[i] = make_uint2((uint32_t)s, (uint32_t)(s >> 32));
-        s_fit[i] = p.fitness[i];
-    }
-    __syncthreads();
-
-    int64_t chunk = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (chunk >= p.n_chunks) return;
+// alone (replay only), selected by p.mode.  Shared memory: 2 * n_pop * 96 B.
+template <int BITS, bool CLAMP_DELTA, bool STATS>
+__global__ void __launch_bounds__(kThreads, QES_MIN_BLOCKS) pass_kernel(PassParams p) {
+    extern __shared__ __align__(16) uint32_t smem[];
     constexpr int T = kCodesPerThread;
-    Chunk<BITS> w;
-    w.load(p.w_in, chunk);
-    float wf[T];
-#pragma unroll
-    for (int t = 0; t < T; ++t) wf[t] = (float)w.get(t);
+    const int64_t chunk = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const bool active = chunk < p.n_chunks;
 
+    Chunk<BITS, kPairs> w;
+    w.clear();
     float e[T];
-    if (p.mode == kStoredResidual) {
-        const float4* r4 = reinterpret_cast<const float4*>(p.residual) + chunk * (T / 4);
 #pragma unroll
-        for (int q = 0; q < T / 4; ++q) {
-            float4 v = r4[q];
-            e[4 * q] = v.x; e[4 * q + 1] = v.y; e[4 * q + 2] = v.z; e[4 * q + 3] = v.w;
+    for (int t = 0; t < T; ++t) e[t] = 0.0f;
+    float nsig24 = 0.0f;
+    PairConst pc[kPairs];
+    uint32_t y = 0u, x0 = 0u;
+    if (active) {
+        w.load(p.w_in, chunk);
+        if (p.mode == kStoredResidual) {
+            const float4* r4 = reinterpret_cast<const float4*>(p.residual) + chunk * (T / 4);
+#pragma unroll
+            for (int q = 0; q < T / 4; ++q) {
+                float4 v = r4[q];
+                e[4 * q] = v.x; e[4 * q + 1] = v.y; e[4 * q + 2] = v.z; e[4 * q + 3] = v.w;
+            }
         }
-    } else {
+        nsig24 = chunk_neg_sigma24(p, chunk);
+        // a thread's pairs share the counter high word: pair0 is a multiple of kPairs
+        const uint64_t pair0 = (p.elem_offset >> 1) + (uint64_t)chunk * kPairs;
+        y = (uint32_t)(pair0 >> 32);
+        x0 = (uint32_t)pair0;
 #pragma unroll
-        for (int t = 0; t < T; ++t) e[t] = 0.0f;
+        for (int i = 0; i < kPairs; ++i) pc[i] = make_pair_const((uint32_t)pair0 + i);
     }
 
-    const float sig = chunk_sigma(p, chunk);
-    const uint64_t pair0 = (p.elem_offset + (uint64_t)chunk * T) >> 1;
-    const uint32_t c0 = (uint32_t)pair0, c1 = (uint32_t)(pair0 >> 32);
     const int last = p.generations - 1;
+    const int buf_words = p.n_pop * kSeedStride;
     unsigned int n_changed = 0, n_blocked_final = 0, n_blocked_replay = 0, n_attempted = 0;
-    Chunk<BITS> out;
+    Chunk<BITS, kPairs> out;
     out.clear();
 
+    if (p.generations > 0) stage_generation(smem, p.seeds, p.fitness, p.n_pop);
     for (int k = 0; k < p.generations; ++k) {
+        __syncthreads();   // generation k is staged; nobody still reads the other buffer
+        if (k < last)
+            stage_generation(smem + ((k + 1) & 1) * buf_words, p.seeds + (int64_t)(k + 1) * p.n_pop,
+                             p.fitness + (int64_t)(k + 1) * p.n_pop, p.n_pop);
+        if (!active) continue;
+        const uint32_t* table = smem + (k & 1) * buf_words;
         float S[T];
 #pragma unroll
         for (int t = 0; t < T; ++t) S[t] = 0.0f;
-        const uint2* keys = s_key + k * p.n_pop;
-        const float* fit = s_fit + k * p.n_pop;
-        for (int i = 0; i < p.n_pop; ++i) {
-            uint2 key = keys[i];
-            float F = fit[i];
-            RoundKeys rk = make_round_keys(key.x, key.y);
+#ifdef QES_SWP
+        // software pipeline over members: the Philox calls of member i+1 are issued next to the
+        // Box-Muller / rounding arithmetic of member i (no dependence between the two)
+        uint32_t rw[kPairs][4];
+        float Fm;
+        {
+            const RoundKeys rk = load_round_keys(table, Fm);
+            const SeedConst sc = make_seed_const(y, rk);
 #pragma unroll
-            for (int pr = 0; pr < T / 2; ++pr) {
-                float d0, d1;
-                delta_pair<CLAMP_DELTA>(c0 + pr, c1, rk, sig, d0, d1);
-                S[2 * pr] = fmaf(F, d0, S[2 * pr]);            // Eq. 5 numerator
-                S[2 * pr + 1] = fmaf(F, d1, S[2 * pr + 1]);
+            for (int pr = 0; pr < kPairs; ++pr) philox_tail(pc[pr], sc, rk, rw[pr][0], rw[pr][1], rw[pr][2], rw[pr][3]);
+        }
+#pragma unroll 1
+        for (int i = 1; i < p.n_pop; ++i) {
+            float Fn;
+            const RoundKeys rk = load_round_keys(table + i * kSeedStride, Fn);
+            const SeedConst sc = make_seed_const(y, rk);
+#pragma unroll
+            for (int pr = 0; pr < kPairs; ++pr) {
+                uint32_t n0, n1, n2, n3;
+                philox_tail(pc[pr], sc, rk, n0, n1, n2, n3);
+                int z0, z1;
+                pair_rounding_sums<CLAMP_DELTA>(rw[pr][0], rw[pr][1], rw[pr][2], rw[pr][3], nsig24, z0, z1);
+                S[2 * pr] = fmaf(Fm, neg_delta_scaled<CLAMP_DELTA>(z0), S[2 * pr]);            // Eq. 5 numerator
+                S[2 * pr + 1] = fmaf(Fm, neg_delta_scaled<CLAMP_DELTA>(z1), S[2 * pr + 1]);
+                rw[pr][0] = n0; rw[pr][1] = n1; rw[pr][2] = n2; rw[pr][3] = n3;
+            }
+            Fm = Fn;
+        }
+#pragma unroll
+        for (int pr = 0; pr < kPairs; ++pr) {
+            int z0, z1;
+            pair_rounding_sums<CLAMP_DELTA>(rw[pr][0], rw[pr][1], rw[pr][2], rw[pr][3], nsig24, z0, z1);
+            S[2 * pr] = fmaf(Fm, neg_delta_scaled<CLAMP_DELTA>(z0), S[2 * pr]);
+            S[2 * pr + 1] = fmaf(Fm, neg_delta_scaled<CLAMP_DELTA>(z1), S[2 * pr + 1]);
+        }
+#else
+#pragma unroll 1
+        for (int i = 0; i < p.n_pop; ++i) {
+            float Fm;   // -F_i * 2^-24
+            const RoundKeys rk = load_round_keys(table + i * kSeedStride, Fm);
+            const SeedConst sc = make_seed_const(y, rk);
+#pragma unroll
+            for (int pr = 0; pr < kPairs; ++pr) {
+                uint32_t r0, r1, r2, r3;
+#ifdef QES_NO_HOIST
+                philox_tail(make_pair_const(x0 + pr), sc, rk, r0, r1, r2, r3);
+#else
+                philox_tail(pc[pr], sc, rk, r0, r1, r2, r3);
+#endif
+                int z0, z1;
+                pair_rounding_sums<CLAMP_DELTA>(r0, r1, r2, r3, nsig24, z0, z1);
+                S[2 * pr] = fmaf(Fm, neg_delta_scaled<CLAMP_DELTA>(z0), S[2 * pr]);            // Eq. 5 numerator
+                S[2 * pr + 1] = fmaf(Fm, neg_delta_scaled<CLAMP_DELTA>(z1), S[2 * pr + 1]);
             }
         }
+#endif
         const bool is_update = (k == last) && (p.mode != kReplayOnly);
 #pragma unroll
         for (int t = 0; t < T; ++t) {
+            float wf = (float)w.get(t);
             float u = fmaf(p.coef, S[t], p.gamma * e[t]);      // Eq. 6
             float step = roundf(u);                            // Eq. 7, half away from zero
-            float applied = applied_step(wf[t], step, p.qmin, p.qmax, p.boundary_mode);
+            float applied = applied_step(wf, step, p.qmin, p.qmax, p.boundary_mode);
             e[t] = u - applied;                                // Eq. 8 with the gated step
-            bool blocked = applied != step;
-            if (is_update) {
-                out.put(t, (int)(wf[t] + applied));
-                n_changed += applied != 0.0f;
-                n_blocked_final += blocked;
-                n_attempted += step != 0.0f;
-            } else {
-                n_blocked_replay += blocked;
+            if (is_update) out.put(t, (int)(wf + applied));
+            if (STATS) {
+                bool blocked = applied != step;
+                if (is_update) {
+                    n_changed += applied != 0.0f;
+                    n_blocked_final += blocked;
+                    n_attempted += step != 0.0f;
+                } else {
+                    n_blocked_replay += blocked;
+                }
             }
         }
     }
 
-    if (p.mode != kReplayOnly) out.store(p.w_out, chunk);
-    if (p.mode != kStateless) {
-        float4* r4 = reinterpret_cast<float4*>(p.residual) + chunk * (T / 4);
+    if (active) {
+        if (p.mode != kReplayOnly) out.store(p.w_out, chunk);
+        if (p.mode != kStateless) {
+            float4* r4 = reinterpret_cast<float4*>(p.residual) + chunk * (T / 4);
 #pragma unroll
-        for (int q = 0; q < T / 4; ++q) r4[q] = make_float4(e[4 * q], e[4 * q + 1], e[4 * q + 2], e[4 * q + 3]);
+            for (int q = 0; q < T / 4; ++q) r4[q] = make_float4(e[4 * q], e[4 * q + 1], e[4 * q + 2], e[4 * q + 3]);
+        }
     }
-    if (p.stats != nullptr) {
-        // the early return above is per thread: reduce over the lanes that are still here
-        unsigned mask = __activemask();
-        n_changed = __reduce_add_sync(mask, n_changed);
-        n_blocked_final = __reduce_add_sync(mask, n_blocked_final);
-        n_blocked_replay = __reduce_add_sync(mask, n_blocked_replay);
-        n_attempted = __reduce_add_sync(mask, n_attempted);
-        if ((threadIdx.x & 31) == (__ffs(mask) - 1)) {
+    if (STATS) {
+        // inactive threads carry zeros: every warp of the CTA is whole here
+        n_changed = __reduce_add_sync(0xffffffffu, n_changed);
+        n_blocked_final = __reduce_add_sync(0xffffffffu, n_blocked_final);
+        n_blocked_replay = __reduce_add_sync(0xffffffffu, n_blocked_replay);
+        n_attempted = __reduce_add_sync(0xffffffffu, n_attempted);
+        if ((threadIdx.x & 31) == 0) {
             if (n_changed) atomicAdd(p.stats + 0, (unsigned long long)n_changed);
             if (n_blocked_final) atomicAdd(p.stats + 1, (unsigned long long)n_blocked_final);
             if (n_blocked_replay) atomicAdd(p.stats + 2, (unsigned long long)n_blocked_replay);
@@ -183,9 +293,20 @@ __global__ void __launch_bounds__(256) pass_kernel(PassParams p) {
     }
 }
 
+// Box-Muller factors of word pairs, for checking the frozen fp32 sequence on its whole domain.
+__global__ void __launch_bounds__(kThreads) gaussian_factors_kernel(const uint32_t* r0, const uint32_t* r1, int64_t n,
+                                                                    float* R, float* C, float* S) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    R[i] = bm_radius(r0[i]);
+    float c, s;
+    bm_cossin(r1[i], c, s);
+    C[i] = c;
+    S[i] = s;
+}
+
 // ------------------------------------------------------------------------- host side
-constexpr int kThreads = 256;
-constexpr size_t kMaxTableBytes = 200 * 1024;   // shared-memory staging limit for (K+1)*N entries
+constexpr size_t kMaxStageBytes = 200 * 1024;   // two generations of staged members must fit in shared memory
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
@@ -197,6 +318,7 @@ int validate(const qes_tensor_desc* d, const qes_hparams* h) {
         return QES_ERR_BAD_SHAPE;
     if (d->elem_offset % 32 != 0) return QES_ERR_BAD_SHAPE;
     if (d->rows > (INT64_MAX / 4) / d->cols) return QES_ERR_BAD_SHAPE;
+    if (d->rows * d->cols / kCodesPerThread > (int64_t)INT32_MAX * kThreads) return QES_ERR_BAD_SHAPE;
     const int lo = -(1 << (d->bits - 1)), hi = (1 << (d->bits - 1)) - 1;
     if (d->qmin >= d->qmax || d->qmin < lo || d->qmax > hi) return QES_ERR_BAD_HPARAM;
     if (!(h->sigma > 0.0f) || !(h->sigma < 1e30f) || h->n_pop <= 0) return QES_ERR_BAD_HPARAM;
@@ -208,7 +330,7 @@ int validate(const qes_tensor_desc* d, const qes_hparams* h) {
 
 PassParams base_params(const qes_tensor_desc* d, const qes_hparams* h, const void* scales) {
     PassParams p{};
-    p.scales = reinterpret_cast<const __half_raw*>(scales);
+    p.scales = reinterpret_cast<const unsigned short*>(scales);
     p.n_chunks = d->rows * d->cols / kCodesPerThread;
     p.cols = d->cols;
     p.elem_offset = d->elem_offset;
@@ -221,6 +343,8 @@ PassParams base_params(const qes_tensor_desc* d, const qes_hparams* h, const voi
     p.gamma = h->gamma;
     p.qmin = (float)d->qmin;
     p.qmax = (float)d->qmax;
+    p.qmin_i = d->qmin;
+    p.qmax_i = d->qmax;
     return p;
 }
 
@@ -230,21 +354,29 @@ bool delta_clamp_needed(const qes_hparams* h) {
     return h->sigma * 5.7682f + 1.0f > 7.0f;
 }
 
-template <int BITS, bool CLAMP>
-int launch_pass(const PassParams& p, size_t smem, cudaStream_t stream) {
+size_t stage_bytes(int n_pop) { return (size_t)2 * (size_t)n_pop * kSeedStride * sizeof(uint32_t); }
+
+template <int BITS, bool CLAMP, bool STATS>
+int launch_pass(const PassParams& p, cudaStream_t stream) {
+    const size_t smem = stage_bytes(p.n_pop);
     if (smem > 48 * 1024) {
-        cudaError_t a = cudaFuncSetAttribute(pass_kernel<BITS, CLAMP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t a = cudaFuncSetAttribute(pass_kernel<BITS, CLAMP, STATS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (a != cudaSuccess) { cudaGetLastError(); return QES_ERR_CUDA; }
     }
     unsigned blocks = (unsigned)((p.n_chunks + kThreads - 1) / kThreads);
-    pass_kernel<BITS, CLAMP><<<blocks, kThreads, smem, stream>>>(p);
+    pass_kernel<BITS, CLAMP, STATS><<<blocks, kThreads, smem, stream>>>(p);
     return cudaGetLastError() == cudaSuccess ? QES_OK : QES_ERR_CUDA;
 }
 
+template <int BITS>
+int dispatch_flags(bool clamp, bool stats, const PassParams& p, cudaStream_t stream) {
+    if (clamp) return stats ? launch_pass<BITS, true, true>(p, stream) : launch_pass<BITS, true, false>(p, stream);
+    return stats ? launch_pass<BITS, false, true>(p, stream) : launch_pass<BITS, false, false>(p, stream);
+}
+
 int dispatch_pass(int bits, bool clamp, const PassParams& p, cudaStream_t stream) {
-    size_t smem = (size_t)p.generations * p.n_pop * (sizeof(uint2) + sizeof(float));
-    if (bits == 4) return clamp ? launch_pass<4, true>(p, smem, stream) : launch_pass<4, false>(p, smem, stream);
-    return clamp ? launch_pass<8, true>(p, smem, stream) : launch_pass<8, false>(p, smem, stream);
+    const bool stats = p.stats != nullptr;
+    return bits == 4 ? dispatch_flags<4>(clamp, stats, p, stream) : dispatch_flags<8>(clamp, stats, p, stream);
 }
 
 int check_table(const uint64_t* seeds, const float* fitness, int64_t generations, int n_pop) {
@@ -252,7 +384,7 @@ int check_table(const uint64_t* seeds, const float* fitness, int64_t generations
         if (seeds == nullptr || fitness == nullptr) return QES_ERR_NULL_PTR;
         if (!aligned(seeds, 8) || !aligned(fitness, 4)) return QES_ERR_MISALIGNED;
     }
-    if ((size_t)generations * (size_t)n_pop * 12 > kMaxTableBytes) return QES_ERR_TOO_LARGE;
+    if (stage_bytes(n_pop) > kMaxStageBytes) return QES_ERR_TOO_LARGE;
     return QES_OK;
 }
 
@@ -274,14 +406,18 @@ int qes_perturb(const qes_tensor_desc* desc, const void* w_in, void* w_out, cons
     p.w_out = w_out;
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
     unsigned blocks = (unsigned)((p.n_chunks + kThreads - 1) / kThreads);
-    uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
+    RoundKeys rk;
+    for (int r = 0; r < 10; ++r) {
+        rk.a[r] = (uint32_t)seed + kPhiloxW0 * (uint32_t)r;
+        rk.b[r] = (uint32_t)(seed >> 32) + kPhiloxW1 * (uint32_t)r;
+    }
     bool clamp = delta_clamp_needed(hparams);
     if (desc->bits == 4) {
-        if (clamp) perturb_kernel<4, true><<<blocks, kThreads, 0, stream>>>(p, k0, k1);
-        else perturb_kernel<4, false><<<blocks, kThreads, 0, stream>>>(p, k0, k1);
+        if (clamp) perturb_kernel<4, true><<<blocks, kThreads, 0, stream>>>(p, rk);
+        else perturb_kernel<4, false><<<blocks, kThreads, 0, stream>>>(p, rk);
     } else {
-        if (clamp) perturb_kernel<8, true><<<blocks, kThreads, 0, stream>>>(p, k0, k1);
-        else perturb_kernel<8, false><<<blocks, kThreads, 0, stream>>>(p, k0, k1);
+        if (clamp) perturb_kernel<8, true><<<blocks, kThreads, 0, stream>>>(p, rk);
+        else perturb_kernel<8, false><<<blocks, kThreads, 0, stream>>>(p, rk);
     }
     return cudaGetLastError() == cudaSuccess ? QES_OK : QES_ERR_CUDA;
 }
@@ -333,6 +469,19 @@ int qes_update(const qes_tensor_desc* desc, void* w_inout, const void* scales_f1
     return dispatch_pass(desc->bits, delta_clamp_needed(hparams), p, reinterpret_cast<cudaStream_t>(cuda_stream));
 }
 
+int qes_gaussian_factors(const uint32_t* r0, const uint32_t* r1, int64_t n, float* radius, float* cosine,
+                         float* sine, void* cuda_stream) {
+    if (n < 0) return QES_ERR_BAD_SHAPE;
+    if (n == 0) return QES_OK;
+    if (r0 == nullptr || r1 == nullptr || radius == nullptr || cosine == nullptr || sine == nullptr) return QES_ERR_NULL_PTR;
+    if (!aligned(r0, 4) || !aligned(r1, 4) || !aligned(radius, 4) || !aligned(cosine, 4) || !aligned(sine, 4))
+        return QES_ERR_MISALIGNED;
+    if ((n + kThreads - 1) / kThreads > (int64_t)INT32_MAX) return QES_ERR_BAD_SHAPE;
+    unsigned blocks = (unsigned)((n + kThreads - 1) / kThreads);
+    gaussian_factors_kernel<<<blocks, kThreads, 0, reinterpret_cast<cudaStream_t>(cuda_stream)>>>(r0, r1, n, radius, cosine, sine);
+    return cudaGetLastError() == cudaSuccess ? QES_OK : QES_ERR_CUDA;
+}
+
 const char* qes_strerror(int status) {
     switch (status) {
         case QES_OK: return "ok";
@@ -343,11 +492,11 @@ const char* qes_strerror(int status) {
         case QES_ERR_BAD_HPARAM: return "hyper-parameter or code range out of bounds";
         case QES_ERR_BAD_MODE: return "unknown mode, or stored residual combined with K > 0";
         case QES_ERR_CUDA: return "CUDA reported an error at launch";
-        case QES_ERR_TOO_LARGE: return "(K+1)*n_pop table exceeds the shared-memory staging limit";
+        case QES_ERR_TOO_LARGE: return "n_pop exceeds the shared-memory staging limit";
         default: return "unknown status";
     }
 }
 
-int qes_version(void) { return 100; }
+int qes_version(void) { return 110; }
 
 }  // extern "C"

@@ -124,6 +124,71 @@ __global__ void __launch_bounds__(kProbeThreads) probe_mix_kernel(int iters, uin
     if (acc == 0x12345u) sink[0] = acc;
 }
 
+// Wide multiplies whose two result halves both stay live (a chain that keeps only the low half
+// can be narrowed by the assembler).  MODE 0: w = lo(w) * a + w, one 64-bit multiply-add per
+// step.  MODE 1: (h, l) = x * a; x = h ^ l ^ b, one wide multiply and one three-input xor per
+// step, the shape of a Philox round.  MODE 2 / 3 / 4: MODE 1 plus one / two / four independent
+// fp32 fused multiply-adds per step, which shows whether fp32 work shares the pipe of the wide
+// multiply or runs beside it.
+template <int MODE>
+__global__ void __launch_bounds__(kProbeThreads) probe_wide_kernel(int iters, uint32_t a, uint32_t b, uint32_t* sink) {
+    constexpr int kFma = MODE == 2 ? 1 : MODE == 3 ? 2 : MODE == 4 ? 4 : 0;
+    unsigned long long w[kChains];
+    float f[kChains][kFma > 0 ? kFma : 1];
+#pragma unroll
+    for (int c = 0; c < kChains; ++c) {
+        w[c] = ((unsigned long long)(threadIdx.x * 2654435761u + c * 40503u) << 32) | (blockIdx.x + 0x3f800001u + c);
+#pragma unroll
+        for (int j = 0; j < (kFma > 0 ? kFma : 1); ++j) f[c][j] = 1.0f + 1e-3f * (float)(threadIdx.x + c + j);
+    }
+    const float fa = __uint_as_float(b), fb = 1e-7f;   // b is passed as the bits of a float just below 1
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int c = 0; c < kChains; ++c) {
+            if (MODE == 0) {
+                asm volatile("mad.wide.u32 %0, %1, %2, %0;" : "+l"(w[c]) : "r"((uint32_t)w[c]), "r"(a));
+            } else {
+                unsigned long long p;
+                asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(p) : "r"((uint32_t)w[c]), "r"(a));
+                w[c] = (uint32_t)(p >> 32) ^ (uint32_t)p ^ b;
+#pragma unroll
+                for (int j = 0; j < kFma; ++j)
+                    asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(f[c][j]) : "f"(fa), "f"(fb));
+            }
+        }
+    }
+    uint32_t acc = 0;
+#pragma unroll
+    for (int c = 0; c < kChains; ++c) {
+        acc ^= (uint32_t)w[c] ^ (uint32_t)(w[c] >> 32);
+#pragma unroll
+        for (int j = 0; j < kFma; ++j) acc ^= __float_as_uint(f[c][j]);
+    }
+    if (acc == 0x12345u) sink[0] = acc;
+}
+
+template <int MODE>
+int run_wide(int iters, uint32_t* sink, float* ms_out, double* ops_out) {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return QES_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return QES_ERR_CUDA;
+    cudaEvent_t e0, e1;
+    cudaEventCreate(&e0); cudaEventCreate(&e1);
+    int blocks = sms * kCtasPerSm;
+    probe_wide_kernel<MODE><<<blocks, kProbeThreads>>>(iters / 8 + 1, 0xD2511F53u, 0x3f7ffff0u, sink);
+    cudaEventRecord(e0);
+    probe_wide_kernel<MODE><<<blocks, kProbeThreads>>>(iters, 0xD2511F53u, 0x3f7ffff0u, sink);
+    cudaEventRecord(e1);
+    cudaError_t err = cudaEventSynchronize(e1);
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, e0, e1);
+    cudaEventDestroy(e0); cudaEventDestroy(e1);
+    if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return QES_ERR_CUDA;
+    *ms_out = ms;
+    *ops_out = (double)blocks * kProbeThreads * (double)iters * (double)kChains;   // steps, not instructions
+    return QES_OK;
+}
+
 template <int KA, int KB>
 int run_mix(int iters, uint32_t* sink, float* ms_out, double* ops_out) {
     int dev = 0, sms = 0;
@@ -194,6 +259,11 @@ extern "C" int qes_pipe_probe(int32_t kind, int32_t iters, void* sink_dev, float
         case 15: return run_probe<15>(iters, sink, ms_out, ops_out);
         case 16: return run_probe<16>(iters, sink, ms_out, ops_out);
         case 17: return run_probe<17>(iters, sink, ms_out, ops_out);
+        case 18: return run_wide<0>(iters, sink, ms_out, ops_out);
+        case 19: return run_wide<1>(iters, sink, ms_out, ops_out);
+        case 20: return run_wide<2>(iters, sink, ms_out, ops_out);
+        case 21: return run_wide<3>(iters, sink, ms_out, ops_out);
+        case 22: return run_wide<4>(iters, sink, ms_out, ops_out);
         case 100: return run_mix<0, 1>(iters, sink, ms_out, ops_out);    // mul.wide + xor3
         case 101: return run_mix<2, 1>(iters, sink, ms_out, ops_out);    // fma + xor3
         case 102: return run_mix<0, 2>(iters, sink, ms_out, ops_out);    // mul.wide + fma

@@ -19,7 +19,8 @@ def lib():
 def test_every_declared_symbol_is_exported(lib):
     header = open(os.path.join(ROOT, "include", "qes.h")).read()
     names = re.findall(r"^(?:int|const char\*)\s+(qes_\w+)\s*\(", header, flags=re.M)
-    assert set(names) >= {"qes_perturb", "qes_update", "qes_replay_residual", "qes_strerror", "qes_version"}
+    assert set(names) >= {"qes_perturb", "qes_update", "qes_replay_residual", "qes_gaussian_factors", "qes_pipe_probe",
+                          "qes_strerror", "qes_version"}
     for n in names:
         assert hasattr(lib, n), n
     assert lib.qes_version() >= 100
@@ -50,7 +51,7 @@ def test_invalid_arguments_are_rejected_without_launching(lib):
     assert call(gamma=1.5) == -5 and call(qmin=3, qmax=3) == -5 and call(qmin=-9, qmax=7) == -5
     assert call(unit=2) == -6 and call(mode=7) == -6 and call(res=0x4000, K=2) == -6
     assert call(w=None) == -1 and call(seeds=None) == -1 and call(unit=1, scales=None) == -1
-    assert call(n_pop=1000, K=100) == -8
+    assert call(n_pop=1067, K=1) == -8 and call(n_pop=1 << 30, K=0) == -8
     d = binding.TensorDesc(bits=4, rows=4, cols=64).c()
     h = binding.HParams(sigma=0.5, lr=1.0, gamma=0.9, n_pop=4).c()
     assert lib.qes_perturb(C.byref(d), None, 0x1000, None, 1, C.byref(h), None) == -1

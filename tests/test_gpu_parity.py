@@ -243,3 +243,19 @@ def test_perturb_delta_is_the_delta_the_update_sums(qo, qes):
     qes.qes_update(tg, w, None, _dev(np.array([[seed]], np.uint64)), _dev(np.array([[1.0]], np.float32)), 0, None, hg)
     assert np.array_equal(_host(wp), _host(w))
     assert np.array_equal(qo.unpack(8, _host(wp), 1024), qo.delta(seed, np.arange(1024, dtype=np.uint64), 1.0)[0])
+
+
+def test_gaussian_factors_bit_identical_on_the_whole_domain(qo, qes):
+    """Every one of the 2^24 radii and 2^24 (cos, sin) pairs of the noise contract: the kernel's fp32
+    sequence (its own square root, its own argument reduction) against the oracle's, bit for bit."""
+    import torch
+    words = (np.arange(1 << 24, dtype=np.uint64) << 8).astype(np.uint32)
+    words |= np.random.default_rng(3).integers(0, 256, size=words.size, dtype=np.uint32)   # low byte is unused
+    w = torch.from_numpy(words.view(np.int32)).cuda()
+    R, Cs, Sn = (torch.empty(words.size, dtype=torch.float32, device="cuda") for _ in range(3))
+    qes.qes_gaussian_factors(w, w, R, Cs, Sn)
+    Ro, Co, So = qo.bm24(words, words)
+    for got, want, name in ((R, Ro, "radius"), (Cs, Co, "cos"), (Sn, So, "sin")):
+        g = _host(got)
+        assert np.array_equal(g.view(np.uint32), want.view(np.uint32)), \
+            f"{name}: {(g.view(np.uint32) != want.view(np.uint32)).sum()} of 2^24 values differ"
