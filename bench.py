@@ -31,13 +31,16 @@ from paper_2602_03120_b200 import workloads as wl  # noqa: E402
 # Algorithmic operation counts of the noise contract (one count per 32-bit multiply, xor, add,
 # shift, conversion, compare/select or fp32 operation the definition requires; square root = 1):
 #   per Philox call (two samples): 10 rounds x (2 wide multiplies + 2 three-input xors)      = 40
-#   Box-Muller pair: uniform 3, log 17, sqrt 1, angle reduction + polynomials + quadrant 19,
-#                    sigma scaling 3                                                          = 43
-#   stochastic rounding, per sample: floor, frac, shift, convert, scale, compare, add, fma = 8 (x2 = 16)
-OPS_PER_SAMPLE = (40 + 43 + 16) / 2.0
+#   Box-Muller pair: radius 20 (uniform 3, log 16, sqrt 1), angle 19 (reduction 7, two
+#                    polynomials 8, quadrant 4), sigma scaling 3                              = 42
+#   Eq. 3 + Eq. 5 per sample: floor, fraction, shift, compare, add, weighted fma = 7 (x2)    = 14
+OPS_PER_SAMPLE = (40 + 42 + 14) / 2.0
 OPS_PER_ELEM_GEN = 8.0      # u (2), round, w + step, two compares, select, residual
 OPS_PER_ELEM = 6.0          # unpack / repack
 SM_COUNT, LANES_PER_SM = 148, 128
+# DRAM bytes of one update launch per algorithmic byte (packed weights read once and written
+# once), from the ncu capture summarised under profiles/; None until a capture of this kernel exists
+DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE = None
 
 
 def alu_ops(numel: int, n_pop: int, generations: int) -> float:
@@ -138,6 +141,7 @@ def config_dict(cfg, n_gpus):
     return {"workload": cfg.name, "bits": cfg.bits, "weights_per_gpu": cfg.numel, "tensors_per_gpu": len(cfg.tensors),
             "n_pop": cfg.n_pop, "K": cfg.K, "sigma": cfg.sigma, "lr": cfg.lr, "gamma": cfg.gamma,
             "sigma_unit": "grid", "boundary": "gate", "perturb_members_per_step": cfg.n_pop,
+            "launches": "one library call per run of consecutive tensors, at most 2^28 codes each",
             "parallelism": f"{n_gpus} x independent shards (no collective)",
             "l2": "weight set (>= 655 MB for the decoder sets) far exceeds the 126 MB L2; "
                   "the 8 MB single-matrix set is flushed by a 256 MB write between steps"}
@@ -200,20 +204,21 @@ def main():
             launches += model.perturb_member(scratch, s)
         if timers is not None:
             b.record(stream)
-        launches += model.update(seeds, fit, cfg.K)             # Algorithm 2
+        n_upd = model.update(seeds, fit, cfg.K)                 # Algorithm 2
         if timers is not None:
             c.record(stream); timers.append((a, b, c))
-        return launches
+        return launches + n_upd, n_upd
 
     for _ in range(args.warmup):
         step()
     barrier()
     sampler = ClockSampler(local); sampler.start()
-    timers, launches = [], 0
+    timers, launches, n_upd_launches = [], 0, 0
     t_begin, t_end = ev(), ev()
     t_begin.record(stream)
     for _ in range(args.steps):
-        launches += step(timers)
+        n_all, n_upd = step(timers)
+        launches += n_all; n_upd_launches += n_upd
     t_end.record(stream)
     barrier()
     clocks = sampler.stop()
@@ -256,17 +261,18 @@ def main():
 
     hbm_gbs, sm_mhz, peak_src = measured_peaks()
     G = cfg.K + 1
-    n_upd_launches = len(model.tensors) * args.steps
-    upd_ops_per_launch = alu_ops(model.numel, cfg.n_pop, G) / len(model.tensors)
+    upd_ops_per_launch = alu_ops(model.numel, cfg.n_pop, G) * args.steps / n_upd_launches
     upd_s_per_launch = update_ms * 1e-3 / n_upd_launches
     alu_peak = SM_COUNT * LANES_PER_SM * sm_mhz * 1e6
     achieved = upd_ops_per_launch / upd_s_per_launch
-    bytes_per_launch = 2 * wl.packed_bytes(cfg.bits, model.numel) / len(model.tensors)
+    bytes_per_launch = 2 * wl.packed_bytes(cfg.bits, model.numel) * args.steps / n_upd_launches
+    traffic = None if DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE is None else DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE * bytes_per_launch
     roofline = {"bound": "alu", "kernel": f"pass_kernel<{cfg.bits}> (qes_update, stateless)",
                 "achieved": achieved / 1e9, "peak": alu_peak / 1e9, "unit": "Glane-op/s", "frac": achieved / alu_peak,
-                "peak_source": f"{SM_COUNT} SMs x 4 schedulers x 32 lanes x {sm_mhz:.0f} MHz (SM clock from {peak_src} peaks file)",
+                "peak_source": f"{SM_COUNT} SMs x 4 schedulers x 32 lanes x {sm_mhz:.0f} MHz (one instruction per scheduler "
+                               f"per cycle; SM clock from the {peak_src} peaks file)",
                 "ops_per_sample": OPS_PER_SAMPLE, "avg_launch_ms": upd_s_per_launch * 1e3, "launches": n_upd_launches,
-                "traffic": None,
+                "traffic": traffic,
                 "hbm": {"achieved_gbs": bytes_per_launch / upd_s_per_launch / 1e9, "peak_gbs": hbm_gbs,
                         "frac": bytes_per_launch / upd_s_per_launch / 1e9 / hbm_gbs, "of": peak_src}}
     line = {"metric": "weights_updated_per_s", "value": value, "unit": "weights/s", "n_gpus": world,

@@ -1,10 +1,12 @@
 // Kernels and C ABI of the QES parameter pass (sm_100a).  See include/qes.h for the contract.
 //
-// Work decomposition: one thread owns 2*kPairs consecutive codes (kPairs Philox calls per seed):
-// with kPairs = 8 a 64-bit load for INT4 and a 128-bit load for INT8, so a warp reads and writes
-// whole 256 B / 512 B segments, once.  Everything else is arithmetic in registers: a code costs
-// one byte of HBM traffic but N*(K+1) noise samples of ~50 operations each, so the kernels are
-// bound by instruction issue and by the integer / wide-multiply pipes, never by memory.
+// Work decomposition: one thread owns 2*kPairs consecutive codes (kPairs Philox calls per seed).
+// With kPairs = 4 that is one 32-bit load for INT4 and one 64-bit load for INT8: a warp reads and
+// writes one contiguous 128 B / 256 B segment, once.  Everything else is arithmetic in
+// registers: a code costs one byte of HBM traffic but N*(K+1) noise samples of ~50 operations
+// each, so the kernels are bound by instruction issue on the multiply and integer pipes, never
+// by memory; kPairs is chosen for the register budget (S, e and the Philox state of 4 pairs fit
+// without spills at two CTAs per SM), not for the width of the load.
 //
 // Per generation the CTA stages, in shared memory, the ten Philox round keys of each of the N
 // seeds next to the member's fitness (96 B per member, double-buffered so one barrier per
@@ -155,7 +157,7 @@ __global__ void __launch_bounds__(kThreads, QES_MIN_BLOCKS) pass_kernel(PassPara
     for (int t = 0; t < T; ++t) e[t] = 0.0f;
     float nsig24 = 0.0f;
     PairConst pc[kPairs];
-    uint32_t y = 0u, x0 = 0u;
+    uint32_t y = 0u;
     if (active) {
         w.load(p.w_in, chunk);
         if (p.mode == kStoredResidual) {
@@ -170,7 +172,6 @@ __global__ void __launch_bounds__(kThreads, QES_MIN_BLOCKS) pass_kernel(PassPara
         // a thread's pairs share the counter high word: pair0 is a multiple of kPairs
         const uint64_t pair0 = (p.elem_offset >> 1) + (uint64_t)chunk * kPairs;
         y = (uint32_t)(pair0 >> 32);
-        x0 = (uint32_t)pair0;
 #pragma unroll
         for (int i = 0; i < kPairs; ++i) pc[i] = make_pair_const((uint32_t)pair0 + i);
     }
@@ -192,42 +193,6 @@ __global__ void __launch_bounds__(kThreads, QES_MIN_BLOCKS) pass_kernel(PassPara
         float S[T];
 #pragma unroll
         for (int t = 0; t < T; ++t) S[t] = 0.0f;
-#ifdef QES_SWP
-        // software pipeline over members: the Philox calls of member i+1 are issued next to the
-        // Box-Muller / rounding arithmetic of member i (no dependence between the two)
-        uint32_t rw[kPairs][4];
-        float Fm;
-        {
-            const RoundKeys rk = load_round_keys(table, Fm);
-            const SeedConst sc = make_seed_const(y, rk);
-#pragma unroll
-            for (int pr = 0; pr < kPairs; ++pr) philox_tail(pc[pr], sc, rk, rw[pr][0], rw[pr][1], rw[pr][2], rw[pr][3]);
-        }
-#pragma unroll 1
-        for (int i = 1; i < p.n_pop; ++i) {
-            float Fn;
-            const RoundKeys rk = load_round_keys(table + i * kSeedStride, Fn);
-            const SeedConst sc = make_seed_const(y, rk);
-#pragma unroll
-            for (int pr = 0; pr < kPairs; ++pr) {
-                uint32_t n0, n1, n2, n3;
-                philox_tail(pc[pr], sc, rk, n0, n1, n2, n3);
-                int z0, z1;
-                pair_rounding_sums<CLAMP_DELTA>(rw[pr][0], rw[pr][1], rw[pr][2], rw[pr][3], nsig24, z0, z1);
-                S[2 * pr] = fmaf(Fm, neg_delta_scaled<CLAMP_DELTA>(z0), S[2 * pr]);            // Eq. 5 numerator
-                S[2 * pr + 1] = fmaf(Fm, neg_delta_scaled<CLAMP_DELTA>(z1), S[2 * pr + 1]);
-                rw[pr][0] = n0; rw[pr][1] = n1; rw[pr][2] = n2; rw[pr][3] = n3;
-            }
-            Fm = Fn;
-        }
-#pragma unroll
-        for (int pr = 0; pr < kPairs; ++pr) {
-            int z0, z1;
-            pair_rounding_sums<CLAMP_DELTA>(rw[pr][0], rw[pr][1], rw[pr][2], rw[pr][3], nsig24, z0, z1);
-            S[2 * pr] = fmaf(Fm, neg_delta_scaled<CLAMP_DELTA>(z0), S[2 * pr]);
-            S[2 * pr + 1] = fmaf(Fm, neg_delta_scaled<CLAMP_DELTA>(z1), S[2 * pr + 1]);
-        }
-#else
 #pragma unroll 1
         for (int i = 0; i < p.n_pop; ++i) {
             float Fm;   // -F_i * 2^-24
@@ -236,18 +201,13 @@ __global__ void __launch_bounds__(kThreads, QES_MIN_BLOCKS) pass_kernel(PassPara
 #pragma unroll
             for (int pr = 0; pr < kPairs; ++pr) {
                 uint32_t r0, r1, r2, r3;
-#ifdef QES_NO_HOIST
-                philox_tail(make_pair_const(x0 + pr), sc, rk, r0, r1, r2, r3);
-#else
                 philox_tail(pc[pr], sc, rk, r0, r1, r2, r3);
-#endif
                 int z0, z1;
                 pair_rounding_sums<CLAMP_DELTA>(r0, r1, r2, r3, nsig24, z0, z1);
                 S[2 * pr] = fmaf(Fm, neg_delta_scaled<CLAMP_DELTA>(z0), S[2 * pr]);            // Eq. 5 numerator
                 S[2 * pr + 1] = fmaf(Fm, neg_delta_scaled<CLAMP_DELTA>(z1), S[2 * pr + 1]);
             }
         }
-#endif
         const bool is_update = (k == last) && (p.mode != kReplayOnly);
 #pragma unroll
         for (int t = 0; t < T; ++t) {

@@ -167,6 +167,67 @@ __global__ void __launch_bounds__(kProbeThreads) probe_wide_kernel(int iters, ui
     if (acc == 0x12345u) sink[0] = acc;
 }
 
+// The instruction mix of the update kernel with full instruction-level parallelism: per step
+// one wide multiply, 2.5 half-rate integer operations (the xor3 of the products plus 1.5
+// independent xor3) and two independent fp32 fused multiply-adds -- by the pipe rates 6 cycles
+// of the multiply pipe, 5 of the integer pipe, 5.5 issue slots.  What this kernel reaches is
+// what a schedule of that mix reaches on the machine.
+__global__ void __launch_bounds__(kProbeThreads) probe_mix_pass_kernel(int iters, uint32_t a, uint32_t b, uint32_t* sink) {
+    constexpr int kC = 4;
+    unsigned long long w[kC];
+    uint32_t u[kC], v[kC];
+    float f[kC][2];
+#pragma unroll
+    for (int c = 0; c < kC; ++c) {
+        w[c] = ((unsigned long long)(threadIdx.x * 2654435761u + c * 40503u) << 32) | (blockIdx.x + 0x3f800001u + c);
+        u[c] = threadIdx.x + 77u * c; v[c] = blockIdx.x + 13u * c;
+        f[c][0] = 1.0f + 1e-3f * (float)(threadIdx.x + c); f[c][1] = 1.0f - 1e-3f * (float)c;
+    }
+    const float fa = __uint_as_float(b), fb = 1e-7f;
+    for (int it = 0; it < iters; it += 2) {
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+#pragma unroll
+            for (int c = 0; c < kC; ++c) {
+                unsigned long long p;
+                asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(p) : "r"((uint32_t)w[c]), "r"(a));
+                w[c] = (uint32_t)(p >> 32) ^ (uint32_t)p ^ b;
+                asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(u[c]) : "r"(a), "r"(b));
+                if (half == 0) asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(v[c]) : "r"(b), "r"(a));
+                asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(f[c][0]) : "f"(fa), "f"(fb));
+                asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(f[c][1]) : "f"(fa), "f"(fb));
+            }
+        }
+    }
+    uint32_t acc = 0;
+#pragma unroll
+    for (int c = 0; c < kC; ++c)
+        acc ^= (uint32_t)w[c] ^ (uint32_t)(w[c] >> 32) ^ u[c] ^ v[c] ^ __float_as_uint(f[c][0]) ^ __float_as_uint(f[c][1]);
+    if (acc == 0x12345u) sink[0] = acc;
+}
+
+int run_mix_pass(int iters, uint32_t* sink, float* ms_out, double* ops_out) {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return QES_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return QES_ERR_CUDA;
+    cudaEvent_t e0, e1;
+    cudaEventCreate(&e0); cudaEventCreate(&e1);
+    int blocks = sms * kCtasPerSm;
+    iters &= ~1;
+    probe_mix_pass_kernel<<<blocks, kProbeThreads>>>(iters / 8 + 2, 0xD2511F53u, 0x3f7ffff0u, sink);
+    cudaEventRecord(e0);
+    probe_mix_pass_kernel<<<blocks, kProbeThreads>>>(iters, 0xD2511F53u, 0x3f7ffff0u, sink);
+    cudaEventRecord(e1);
+    cudaError_t err = cudaEventSynchronize(e1);
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, e0, e1);
+    cudaEventDestroy(e0); cudaEventDestroy(e1);
+    if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return QES_ERR_CUDA;
+    *ms_out = ms;
+    *ops_out = (double)blocks * kProbeThreads * (double)iters * 4.0;   // steps (one wide multiply each)
+    return QES_OK;
+}
+
 template <int MODE>
 int run_wide(int iters, uint32_t* sink, float* ms_out, double* ops_out) {
     int dev = 0, sms = 0;
@@ -264,6 +325,7 @@ extern "C" int qes_pipe_probe(int32_t kind, int32_t iters, void* sink_dev, float
         case 20: return run_wide<2>(iters, sink, ms_out, ops_out);
         case 21: return run_wide<3>(iters, sink, ms_out, ops_out);
         case 22: return run_wide<4>(iters, sink, ms_out, ops_out);
+        case 23: return run_mix_pass(iters, sink, ms_out, ops_out);
         case 100: return run_mix<0, 1>(iters, sink, ms_out, ops_out);    // mul.wide + xor3
         case 101: return run_mix<2, 1>(iters, sink, ms_out, ops_out);    // fma + xor3
         case 102: return run_mix<0, 2>(iters, sink, ms_out, ops_out);    // mul.wide + fma

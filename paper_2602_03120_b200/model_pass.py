@@ -1,8 +1,9 @@
 """A whole weight set on one GPU: flat packed buffer, per-tensor descriptors, and the three passes.
 
 This is the call a user of the library makes for a model: ``perturb_member`` (Algorithm 1, member
-loop), ``update`` (Algorithm 2) and ``replay_residual`` launch one library call per tensor on the
-current stream.  Nothing here computes: every step runs in the kernels behind the C ABI.
+loop), ``update`` (Algorithm 2) and ``replay_residual`` launch one library call per tensor -- or, when
+sigma is in grid units and the kernels need no per-tensor geometry, per run of consecutive tensors
+-- on the current stream.  Nothing here computes: every step runs in the kernels behind the C ABI.
 """
 from __future__ import annotations
 
@@ -22,12 +23,33 @@ def shard_tensors(workload: wl.Workload, rank: int, world: int):
                  for t in workload.tensors)
 
 
+MAX_SEGMENT_ELEMS = 1 << 28   # one launch covers at most this many codes (a few hundred ms of work)
+
+
+def launch_segments(tensors, max_elems: int = MAX_SEGMENT_ELEMS):
+    """Groups consecutive tensors into launches of at most `max_elems` codes.  With sigma in grid
+    units the kernels never look at rows, columns or scales: noise depends only on the global
+    element index, so any contiguous run of tensors can be passed as one [numel / 32, 32] tensor.
+    Returns (first_tensor_index, elem_offset, numel) triples; a tensor larger than the limit is a
+    segment of its own."""
+    segs, start, off, n = [], 0, None, 0
+    for i, t in enumerate(tensors):
+        if n and (n + t.numel > max_elems or t.elem_offset != off + n):
+            segs.append((start, off, n)); n = 0
+        if n == 0:
+            start, off = i, t.elem_offset
+        n += t.numel
+    if n:
+        segs.append((start, off, n))
+    return segs
+
+
 class ModelPass:
     def __init__(self, workload: wl.Workload, device="cuda", rank: int = 0, world: int = 1,
-                 sigma_unit: int = qes.SIGMA_GRID, with_scales: bool = False):
+                 sigma_unit: int = qes.SIGMA_GRID, with_scales: bool = False, tensors=None):
         self.wl = workload
         self.device = torch.device(device)
-        self.tensors = shard_tensors(workload, rank, world)
+        self.tensors = tuple(tensors) if tensors is not None else shard_tensors(workload, rank, world)
         self.base = self.tensors[0].elem_offset
         self.numel = sum(t.numel for t in self.tensors)
         self.bytes = wl.packed_bytes(workload.bits, self.numel)
@@ -36,6 +58,11 @@ class ModelPass:
                               sigma_unit=sigma_unit)
         self.descs = [qes.TensorDesc(bits=workload.bits, rows=t.rows, cols=t.cols, group_size=workload.group_size,
                                      elem_offset=t.elem_offset) for t in self.tensors]
+        # grid-unit sigma: fused launches over runs of tensors; weight-unit sigma: one launch per tensor
+        self.fused = sigma_unit == qes.SIGMA_GRID
+        self.segments = [(wl.TensorSpec(f"segment{j}", n // 32, 32, off),
+                          qes.TensorDesc(bits=workload.bits, rows=n // 32, cols=32, group_size=0, elem_offset=off))
+                         for j, (_, off, n) in enumerate(launch_segments(self.tensors))]
         self.scales = None
         if with_scales or sigma_unit == qes.SIGMA_WEIGHT:
             self.scales = [torch.from_numpy(wl.draw_scales(workload, i)).to(self.device)
@@ -60,19 +87,27 @@ class ModelPass:
     def _sc(self, i):
         return None if self.scales is None else self.scales[i]
 
+    def _launches(self):
+        """(tensor spec, descriptor, scales) per library call."""
+        if self.fused:
+            return [(t, d, None) for t, d in self.segments]
+        return [(t, d, self._sc(i)) for i, (t, d) in enumerate(zip(self.tensors, self.descs))]
+
     def perturb_member(self, out: torch.Tensor, seed: int) -> int:
-        for i, (t, d) in enumerate(zip(self.tensors, self.descs)):
-            qes.qes_perturb(d, self._slice(self.w, t), self._slice(out, t), self._sc(i), seed, self.hp)
-        return len(self.tensors)
+        calls = self._launches()
+        for t, d, sc in calls:
+            qes.qes_perturb(d, self._slice(self.w, t), self._slice(out, t), sc, seed, self.hp)
+        return len(calls)
 
     def update(self, seeds: torch.Tensor, fitness: torch.Tensor, K: int, stats=None) -> int:
-        for i, (t, d) in enumerate(zip(self.tensors, self.descs)):
-            qes.qes_update(d, self._slice(self.w, t), self._sc(i), seeds, fitness, K, None, self.hp, stats=stats)
-        return len(self.tensors)
+        calls = self._launches()
+        for t, d, sc in calls:
+            qes.qes_update(d, self._slice(self.w, t), sc, seeds, fitness, K, None, self.hp, stats=stats)
+        return len(calls)
 
     def replay_residual(self, seeds: torch.Tensor, fitness: torch.Tensor, K: int, out: torch.Tensor) -> int:
-        for i, (t, d) in enumerate(zip(self.tensors, self.descs)):
+        calls = self._launches()
+        for t, d, sc in calls:
             lo = t.elem_offset - self.base
-            qes.qes_replay_residual(d, self._slice(self.w, t), self._sc(i), seeds, fitness, K, self.hp,
-                                    out[lo:lo + t.numel])
-        return len(self.tensors)
+            qes.qes_replay_residual(d, self._slice(self.w, t), sc, seeds, fitness, K, self.hp, out[lo:lo + t.numel])
+        return len(calls)

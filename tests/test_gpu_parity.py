@@ -259,3 +259,35 @@ def test_gaussian_factors_bit_identical_on_the_whole_domain(qo, qes):
         g = _host(got)
         assert np.array_equal(g.view(np.uint32), want.view(np.uint32)), \
             f"{name}: {(g.view(np.uint32) != want.view(np.uint32)).sum()} of 2^24 values differ"
+
+
+def test_fused_launch_segments_match_per_tensor_oracle(qo, qes):
+    """The whole-model pass the benchmark times: runs of consecutive tensors go to the library as one
+    [numel / 32, 32] tensor (at most 2^28 codes per call).  Checked on the first two layers of the 7B-shaped
+    INT4 set (14 tensors, two segments) against the oracle run tensor by tensor with each tensor's own
+    geometry, on sampled words that include both ends of every tensor."""
+    from paper_2602_03120_b200.model_pass import ModelPass, launch_segments
+    cfg = wl.WORKLOADS["decoder7b_int4"]
+    tensors = cfg.tensors[:14]
+    model = ModelPass(cfg, tensors=tensors)
+    assert len(model.segments) == len(launch_segments(tensors)) == 2
+    assert sum(t.numel for t, _ in model.segments) == sum(t.numel for t in tensors)
+    host = model.host_codes()
+    model.load(host)
+    seeds, fit = wl.draw_seeds(cfg.K + 1, cfg.n_pop), wl.draw_fitness(cfg.K + 1, cfg.n_pop, cfg.reward_dist)
+    assert model.update(_dev(seeds), _dev(fit), cfg.K) == 2
+    got_all = _host(model.w)
+    ho = qo.HParams(sigma=cfg.sigma, lr=cfg.lr, gamma=cfg.gamma, n_pop=cfg.n_pop)
+    near_total = 0
+    for ti, t in enumerate(tensors):
+        lo = t.elem_offset // 2
+        packed = host[lo:lo + t.numel // 2]
+        assert np.array_equal(packed, wl.draw_codes(cfg, ti))
+        to = qo.Tensor(bits=4, rows=t.rows, cols=t.cols, group_size=cfg.group_size, elem_offset=t.elem_offset)
+        idx = wl.sample_elements(t.numel, 512, stream=100 + ti)
+        ref = qo.update(to, packed, None, seeds, fit, cfg.K, ho, idx=idx)
+        got = qo.unpack(4, got_all[lo:lo + t.numel // 2], t.numel)[idx]
+        near = ref["band"] < BAND
+        assert not np.any((got != ref["w_new"]) & ~near), f"tensor {ti} ({t.name})"
+        near_total += int(near.sum())
+    print(f"fused segments: near-band sampled elements {near_total}")
