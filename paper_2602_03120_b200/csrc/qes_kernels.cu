@@ -31,7 +31,7 @@ enum PassMode : int { kStateless = 0, kStoredResidual = 1, kReplayOnly = 2 };
 constexpr int kThreads = 256;
 constexpr int kPairs = QES_PAIRS;
 constexpr int kCodesPerThread = 2 * kPairs;
-constexpr int kSeedStride = 24;   // 32-bit words per staged member: a[10], b[10], fitness, 3 pad
+constexpr int kSeedStride = 24;   // 32-bit words per staged member: a[10], b[10], fitness, SeedConst
 
 struct PassParams {
     const void* w_in;
@@ -113,25 +113,29 @@ __global__ void __launch_bounds__(kThreads) perturb_kernel(PassParams p, RoundKe
 }
 
 // Expands the seeds of one generation into round keys, next to the fitness values (stored as
-// -F * 2^-24, the factor that turns the kernel's -delta * 2^24 back into F * delta).
-__device__ __forceinline__ void stage_generation(uint32_t* buf, const uint64_t* seeds, const float* fitness, int n_pop) {
+// -F * 2^-24, the factor that turns the kernel's -delta * 2^24 back into F * delta) and the
+// seed's SeedConst for counter high word y_cta (the one almost every CTA has throughout).
+__device__ __forceinline__ void stage_generation(uint32_t* buf, const uint64_t* seeds, const float* fitness, int n_pop,
+                                                 uint32_t y_cta) {
     for (int i = threadIdx.x; i < n_pop; i += kThreads) {
         uint64_t s = seeds[i];
         RoundKeys rk = make_round_keys((uint32_t)s, (uint32_t)(s >> 32));
+        SeedConst sc = make_seed_const(y_cta, rk);
         uint4* d = reinterpret_cast<uint4*>(buf + i * kSeedStride);
         d[0] = make_uint4(rk.a[0], rk.a[1], rk.a[2], rk.a[3]);
         d[1] = make_uint4(rk.a[4], rk.a[5], rk.a[6], rk.a[7]);
         d[2] = make_uint4(rk.a[8], rk.a[9], rk.b[0], rk.b[1]);
         d[3] = make_uint4(rk.b[2], rk.b[3], rk.b[4], rk.b[5]);
         d[4] = make_uint4(rk.b[6], rk.b[7], rk.b[8], rk.b[9]);
-        d[5] = make_uint4(__float_as_uint(fitness[i] * -0x1p-24f), 0u, 0u, 0u);   // pairs with -delta * 2^24
+        d[5] = make_uint4(__float_as_uint(fitness[i] * -0x1p-24f), sc.hak, sc.la, sc.lak);   // pairs with -delta * 2^24
     }
 }
 
-__device__ __forceinline__ RoundKeys load_round_keys(const uint32_t* entry, float& fit) {
+__device__ __forceinline__ RoundKeys load_round_keys(const uint32_t* entry, float& fit, SeedConst& sc) {
     const uint4* q = reinterpret_cast<const uint4*>(entry);
-    uint4 k0 = q[0], k1 = q[1], k2 = q[2], k3 = q[3], k4 = q[4];
-    fit = __uint_as_float(entry[20]);
+    uint4 k0 = q[0], k1 = q[1], k2 = q[2], k3 = q[3], k4 = q[4], k5 = q[5];
+    fit = __uint_as_float(k5.x);
+    sc.hak = k5.y; sc.la = k5.z; sc.lak = k5.w;
     RoundKeys rk;
     rk.a[0] = k0.x; rk.a[1] = k0.y; rk.a[2] = k0.z; rk.a[3] = k0.w;
     rk.a[4] = k1.x; rk.a[5] = k1.y; rk.a[6] = k1.z; rk.a[7] = k1.w;
@@ -182,12 +186,18 @@ __global__ void __launch_bounds__(kThreads, QES_MIN_BLOCKS) pass_kernel(PassPara
     Chunk<BITS, kPairs> out;
     out.clear();
 
-    if (p.generations > 0) stage_generation(smem, p.seeds, p.fitness, p.n_pop);
+    // counter high word of the CTA's first pair; a CTA spans 256 * kPairs pairs, so at most one
+    // CTA in 2^32 / (256 * kPairs) sees a second value, and then its threads rebuild SeedConst
+    const uint64_t cta_pair0 = (p.elem_offset >> 1) + (uint64_t)blockIdx.x * (kThreads * kPairs);
+    const uint32_t y_cta = (uint32_t)(cta_pair0 >> 32);
+    const bool y_uniform = (uint32_t)((cta_pair0 + (uint64_t)(kThreads * kPairs - 1)) >> 32) == y_cta;
+
+    if (p.generations > 0) stage_generation(smem, p.seeds, p.fitness, p.n_pop, y_cta);
     for (int k = 0; k < p.generations; ++k) {
         __syncthreads();   // generation k is staged; nobody still reads the other buffer
         if (k < last)
             stage_generation(smem + ((k + 1) & 1) * buf_words, p.seeds + (int64_t)(k + 1) * p.n_pop,
-                             p.fitness + (int64_t)(k + 1) * p.n_pop, p.n_pop);
+                             p.fitness + (int64_t)(k + 1) * p.n_pop, p.n_pop, y_cta);
         if (!active) continue;
         const uint32_t* table = smem + (k & 1) * buf_words;
         float S[T];
@@ -196,8 +206,9 @@ __global__ void __launch_bounds__(kThreads, QES_MIN_BLOCKS) pass_kernel(PassPara
 #pragma unroll 1
         for (int i = 0; i < p.n_pop; ++i) {
             float Fm;   // -F_i * 2^-24
-            const RoundKeys rk = load_round_keys(table + i * kSeedStride, Fm);
-            const SeedConst sc = make_seed_const(y, rk);
+            SeedConst sc;
+            const RoundKeys rk = load_round_keys(table + i * kSeedStride, Fm, sc);
+            if (!y_uniform) sc = make_seed_const(y, rk);
 #pragma unroll
             for (int pr = 0; pr < kPairs; ++pr) {
                 uint32_t r0, r1, r2, r3;

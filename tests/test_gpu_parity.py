@@ -291,3 +291,20 @@ def test_fused_launch_segments_match_per_tensor_oracle(qo, qes):
         assert not np.any((got != ref["w_new"]) & ~near), f"tensor {ti} ({t.name})"
         near_total += int(near.sum())
     print(f"fused segments: near-band sampled elements {near_total}")
+
+
+@pytest.mark.parametrize("bits,off", [(4, (1 << 33) - 1024), (8, (1 << 33) - 32), (4, (1 << 33) - 2048)])
+def test_update_where_the_counter_high_word_changes(qo, qes, bits, off):
+    """Element 2^33 is where the high word of the Philox counter (pair index >> 32) steps from 0 to 1:
+    a tensor that straddles it (inside a thread block, at a block edge, one word before it)."""
+    rows, cols, N, K = 12, 512, 5, 2
+    to, tg, packed, _ = _case(qo, qes, bits, rows, cols, off=off)
+    ho, hg = _hp(qo, qes, sigma=0.5, lr=1.0, gamma=0.9, n_pop=N)
+    seeds, fit = wl.draw_seeds(K + 1, N, stream=33), wl.draw_fitness(K + 1, N, stream=33)
+    w = _dev(packed)
+    qes.qes_update(tg, w, None, _dev(seeds), _dev(fit), K, None, hg)
+    ref = qo.update(to, packed, None, seeds, fit, K, ho)
+    _compare_update(qo, _host(w), bits, ref, "counter high word")
+    wp = _dev(np.zeros_like(packed))
+    qes.qes_perturb(tg, _dev(packed), wp, None, int(seeds[0, 0]), hg)
+    assert np.array_equal(_host(wp), qo.pack(bits, qo.perturb(to, packed, None, int(seeds[0, 0]), ho)))
