@@ -171,7 +171,9 @@ __global__ void __launch_bounds__(kProbeThreads) probe_wide_kernel(int iters, ui
 // one wide multiply, 2.5 half-rate integer operations (the xor3 of the products plus 1.5
 // independent xor3) and two independent fp32 fused multiply-adds -- by the pipe rates 6 cycles
 // of the multiply pipe, 5 of the integer pipe, 5.5 issue slots.  What this kernel reaches is
-// what a schedule of that mix reaches on the machine.
+// what a schedule of that mix reaches on the machine.  ORDER sets the program order of the
+// instructions inside a step: 0 chain by chain, 1 kinds alternating, 2 kinds grouped.
+template <int ORDER>
 __global__ void __launch_bounds__(kProbeThreads) probe_mix_pass_kernel(int iters, uint32_t a, uint32_t b, uint32_t* sink) {
     constexpr int kC = 4;
     unsigned long long w[kC];
@@ -187,15 +189,57 @@ __global__ void __launch_bounds__(kProbeThreads) probe_mix_pass_kernel(int iters
     for (int it = 0; it < iters; it += 2) {
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
+            if (ORDER == 0) {          // per chain: wide, its xor3, the independent xor3s, the two fmas
 #pragma unroll
-            for (int c = 0; c < kC; ++c) {
-                unsigned long long p;
-                asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(p) : "r"((uint32_t)w[c]), "r"(a));
-                w[c] = (uint32_t)(p >> 32) ^ (uint32_t)p ^ b;
-                asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(u[c]) : "r"(a), "r"(b));
-                if (half == 0) asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(v[c]) : "r"(b), "r"(a));
-                asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(f[c][0]) : "f"(fa), "f"(fb));
-                asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(f[c][1]) : "f"(fa), "f"(fb));
+                for (int c = 0; c < kC; ++c) {
+                    unsigned long long p;
+                    asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(p) : "r"((uint32_t)w[c]), "r"(a));
+                    asm volatile("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(u[c]) : "r"(u[c]), "r"(a), "r"(b));
+                    uint32_t x;
+                    asm volatile("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(x) : "r"((uint32_t)(p >> 32)), "r"((uint32_t)p), "r"(b));
+                    w[c] = x;
+                    if (half == 0) asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(v[c]) : "r"(b), "r"(a));
+                    asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(f[c][0]) : "f"(fa), "f"(fb));
+                    asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(f[c][1]) : "f"(fa), "f"(fb));
+                }
+            } else if (ORDER == 1) {   // kinds alternate: wide, fma, xor3, fma, xor3 (+ xor3)
+                unsigned long long p[kC];
+#pragma unroll
+                for (int c = 0; c < kC; ++c) {
+                    asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(p[c]) : "r"((uint32_t)w[c]), "r"(a));
+                    asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(f[c][0]) : "f"(fa), "f"(fb));
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(u[c]) : "r"(a), "r"(b));
+                    asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(f[c][1]) : "f"(fa), "f"(fb));
+                    if (half == 0) asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(v[c]) : "r"(b), "r"(a));
+                    if (c > 0) {
+                        uint32_t x;
+                        asm volatile("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(x) : "r"((uint32_t)(p[c - 1] >> 32)), "r"((uint32_t)p[c - 1]), "r"(b));
+                        w[c - 1] = x;
+                    }
+                }
+                uint32_t x;
+                asm volatile("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(x) : "r"((uint32_t)(p[kC - 1] >> 32)), "r"((uint32_t)p[kC - 1]), "r"(b));
+                w[kC - 1] = x;
+            } else {                   // kinds grouped: all wides, all xor3s, all fmas
+                unsigned long long p[kC];
+#pragma unroll
+                for (int c = 0; c < kC; ++c) asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(p[c]) : "r"((uint32_t)w[c]), "r"(a));
+#pragma unroll
+                for (int c = 0; c < kC; ++c) {
+                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(u[c]) : "r"(a), "r"(b));
+                    if (half == 0) asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(v[c]) : "r"(b), "r"(a));
+                }
+#pragma unroll
+                for (int c = 0; c < kC; ++c) {
+                    uint32_t x;
+                    asm volatile("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(x) : "r"((uint32_t)(p[c] >> 32)), "r"((uint32_t)p[c]), "r"(b));
+                    w[c] = x;
+                }
+#pragma unroll
+                for (int c = 0; c < kC; ++c) {
+                    asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(f[c][0]) : "f"(fa), "f"(fb));
+                    asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(f[c][1]) : "f"(fa), "f"(fb));
+                }
             }
         }
     }
@@ -206,6 +250,7 @@ __global__ void __launch_bounds__(kProbeThreads) probe_mix_pass_kernel(int iters
     if (acc == 0x12345u) sink[0] = acc;
 }
 
+template <int ORDER>
 int run_mix_pass(int iters, uint32_t* sink, float* ms_out, double* ops_out) {
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return QES_ERR_CUDA;
@@ -214,9 +259,9 @@ int run_mix_pass(int iters, uint32_t* sink, float* ms_out, double* ops_out) {
     cudaEventCreate(&e0); cudaEventCreate(&e1);
     int blocks = sms * kCtasPerSm;
     iters &= ~1;
-    probe_mix_pass_kernel<<<blocks, kProbeThreads>>>(iters / 8 + 2, 0xD2511F53u, 0x3f7ffff0u, sink);
+    probe_mix_pass_kernel<ORDER><<<blocks, kProbeThreads>>>(iters / 8 + 2, 0xD2511F53u, 0x3f7ffff0u, sink);
     cudaEventRecord(e0);
-    probe_mix_pass_kernel<<<blocks, kProbeThreads>>>(iters, 0xD2511F53u, 0x3f7ffff0u, sink);
+    probe_mix_pass_kernel<ORDER><<<blocks, kProbeThreads>>>(iters, 0xD2511F53u, 0x3f7ffff0u, sink);
     cudaEventRecord(e1);
     cudaError_t err = cudaEventSynchronize(e1);
     float ms = 0.f;
@@ -325,7 +370,9 @@ extern "C" int qes_pipe_probe(int32_t kind, int32_t iters, void* sink_dev, float
         case 20: return run_wide<2>(iters, sink, ms_out, ops_out);
         case 21: return run_wide<3>(iters, sink, ms_out, ops_out);
         case 22: return run_wide<4>(iters, sink, ms_out, ops_out);
-        case 23: return run_mix_pass(iters, sink, ms_out, ops_out);
+        case 23: return run_mix_pass<0>(iters, sink, ms_out, ops_out);
+        case 24: return run_mix_pass<1>(iters, sink, ms_out, ops_out);
+        case 25: return run_mix_pass<2>(iters, sink, ms_out, ops_out);
         case 100: return run_mix<0, 1>(iters, sink, ms_out, ops_out);    // mul.wide + xor3
         case 101: return run_mix<2, 1>(iters, sink, ms_out, ops_out);    // fma + xor3
         case 102: return run_mix<0, 2>(iters, sink, ms_out, ops_out);    // mul.wide + fma
