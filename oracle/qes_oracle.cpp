@@ -105,14 +105,16 @@ void bm24_cossin(uint32_t r1, float* c_out, float* s_out) {
 // with the 24-bit uniform v = (word >> 8) / 2^24.  x is the fp32 value sigma_eff * eps; its
 // fractional part and the comparison are evaluated exactly (both are exact in double), so
 // P(b = 1) is the fractional part of x to within the 2^-24 grid of v and nothing else.  Then the
-// 4-bit range of the perturbation tensor (App. A "4-bit stochastically rounded perturbation").
-int stochastic_round_f32(float x, uint32_t rword) {
+// 4-bit range of the perturbation tensor (App. A "4-bit stochastically rounded perturbation"):
+// [-8, 7], or the symmetric [-7, 7] (dmin = -7) when members come in antithetic pairs +-delta,
+// so that the mirrored member fits the same 4 bits.
+int stochastic_round_f32(float x, uint32_t rword, int dmin = -8) {
     double xd = (double)x;
     double fl = std::floor(xd);
     double frac = xd - fl;                          // exact
     double v = (double)(rword >> 8) / 16777216.0;   // exact, [0,1)
     int d = (int)fl + (v < frac ? 1 : 0);
-    return std::min(7, std::max(-8, d));
+    return std::min(7, std::max(dmin, d));
 }
 
 struct PairNoise { int delta[2]; double x[2]; bool near[2]; };
@@ -122,7 +124,7 @@ const double kPi = 3.14159265358979323846;
 // Both discrete perturbations of pair p for one seed.  sig[] = sigma_eff of the
 // even and odd element.  tier 0 also flags samples whose decision lies within
 // tau of a floor boundary or of the Bernoulli threshold.
-PairNoise pair_noise(uint64_t seed, uint64_t p, const float sig[2], int tier, double tau) {
+PairNoise pair_noise(uint64_t seed, uint64_t p, const float sig[2], int tier, double tau, int dmin = -8) {
     U4 r = philox4x32_10((uint32_t)p, (uint32_t)(p >> 32), 0u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32));
     PairNoise out;
     if (tier == 1) {
@@ -133,7 +135,7 @@ PairNoise pair_noise(uint64_t seed, uint64_t p, const float sig[2], int tier, do
         for (int h = 0; h < 2; ++h) {
             float rho = sig[h] * R;
             float x = rho * trig[h];
-            out.delta[h] = stochastic_round_f32(x, r.v[2 + h]);
+            out.delta[h] = stochastic_round_f32(x, r.v[2 + h], dmin);
             out.x[h] = (double)x;
             out.near[h] = false;
         }
@@ -149,7 +151,7 @@ PairNoise pair_noise(uint64_t seed, uint64_t p, const float sig[2], int tier, do
             double frac = x - fl;
             double v = (double)(r.v[2 + h] >> 8) / 16777216.0;
             int d = (int)fl + (v < frac ? 1 : 0);
-            out.delta[h] = std::min(7, std::max(-8, d));
+            out.delta[h] = std::min(7, std::max(dmin, d));
             out.x[h] = x;
             out.near[h] = (frac < tau) || (frac > 1.0 - tau) || (std::fabs(frac - v) < tau);
         }
@@ -188,7 +190,10 @@ void store_code(uint8_t* packed, int bits, int64_t j, int code) {
 }
 
 struct Tensor { int32_t bits, qmin, qmax, group_size; int64_t rows, cols; uint64_t elem_offset; };
-struct HParams { float sigma, lr, gamma; int32_t n_pop, sigma_unit, boundary_mode; };
+// antithetic != 0 (App. A "antithetic perturbation pairs"): the population is n_pop / 2 pairs, pair j
+// has one seed and the two members W + delta_j and W - delta_j; seeds hold n_pop / 2 entries per
+// generation, fitness holds n_pop entries per generation ordered F+_0, F-_0, F+_1, F-_1, ...
+struct HParams { float sigma, lr, gamma; int32_t n_pop, sigma_unit, boundary_mode, antithetic; };
 
 float sigma_eff(const Tensor& t, const HParams& hp, const uint16_t* scales, int64_t j) {
     if (hp.sigma_unit == 0) return hp.sigma;                    // sigma in grid steps
@@ -210,6 +215,8 @@ int check(const Tensor& t, const HParams& hp) {
     if (t.rows <= 0 || t.cols <= 0 || (t.cols & 1)) return -3;
     if (t.group_size < 0 || (t.group_size > 0 && t.cols % t.group_size)) return -3;
     if (!(hp.sigma > 0.f) || hp.n_pop <= 0 || !(hp.gamma >= 0.f && hp.gamma <= 1.f) || t.qmin >= t.qmax) return -5;
+    if (hp.antithetic != 0 && hp.antithetic != 1) return -6;
+    if (hp.antithetic && (hp.n_pop & 1)) return -5;
     return 0;
 }
 
@@ -245,9 +252,18 @@ ElemResult element_update(const Tensor& t, const HParams& hp, const uint16_t* sc
     double e = e0;
     for (int k = 0; k < gens; ++k) {
         double S = 0.0;
-        for (int i = 0; i < N; ++i) {
-            PairNoise pn = pair_noise(seeds[(int64_t)k * N + i], p, sig, tier, 0.0);
-            S += (double)fitness[(int64_t)k * N + i] * (double)pn.delta[h];   // Eq. 5 numerator
+        if (!hp.antithetic) {
+            for (int i = 0; i < N; ++i) {
+                PairNoise pn = pair_noise(seeds[(int64_t)k * N + i], p, sig, tier, 0.0);
+                S += (double)fitness[(int64_t)k * N + i] * (double)pn.delta[h];   // Eq. 5 numerator
+            }
+        } else {
+            // Eq. 5 over all N members, members 2j and 2j+1 carrying +delta_j and -delta_j
+            for (int jp = 0; jp < N / 2; ++jp) {
+                PairNoise pn = pair_noise(seeds[(int64_t)k * (N / 2) + jp], p, sig, tier, 0.0, -7);
+                S += (double)fitness[(int64_t)k * N + 2 * jp] * (double)pn.delta[h];
+                S += (double)fitness[(int64_t)k * N + 2 * jp + 1] * (double)(-pn.delta[h]);
+            }
         }
         double u = c * S + gamma * e;                                          // Eq. 6
         double step = std::round(u);                                           // Eq. 7, half away from zero
@@ -292,11 +308,11 @@ float qo_half_to_float(uint16_t h) { return half_to_float(h); }
 
 // delta (and optionally x = sigma_eff * eps, near-decision flags) of global
 // elements J[0..n) for one seed and one sigma_eff.
-void qo_delta(uint64_t seed, const uint64_t* J, int64_t n, float sigma_eff_v, int tier, double tau,
+void qo_delta(uint64_t seed, const uint64_t* J, int64_t n, float sigma_eff_v, int tier, double tau, int dmin,
               int32_t* delta, double* x, uint8_t* near) {
     float sig[2] = {sigma_eff_v, sigma_eff_v};
     for (int64_t i = 0; i < n; ++i) {
-        PairNoise pn = pair_noise(seed, J[i] >> 1, sig, tier, tau);
+        PairNoise pn = pair_noise(seed, J[i] >> 1, sig, tier, tau, dmin);
         int h = (int)(J[i] & 1);
         delta[i] = pn.delta[h];
         if (x) x[i] = pn.x[h];
@@ -316,7 +332,8 @@ long long qo_applied_step(int w, long long step, int qmin, int qmax, int mode) {
 
 // Algorithm 1, lines "Reconstruct delta_i" and "Gate(W + delta_i)" for one member.
 // idx == NULL: elements 0..n-1.  w_out[i] = perturbed code of element idx[i].
-int qo_perturb(const Tensor* t, const uint8_t* w, const uint16_t* scales, uint64_t seed,
+// sign = +1: W + delta; sign = -1: the antithetic member W - delta (App. A).
+int qo_perturb(const Tensor* t, const uint8_t* w, const uint16_t* scales, uint64_t seed, int sign,
                const HParams* hp, int tier, const int64_t* idx, int64_t n, int nthreads, int32_t* w_out) {
     int rc = check(*t, *hp);
     if (rc) return rc;
@@ -327,9 +344,9 @@ int qo_perturb(const Tensor* t, const uint8_t* w, const uint16_t* scales, uint64
             int h = (int)(J & 1);
             float sig[2];
             sig[0] = sig[1] = sigma_eff(*t, *hp, scales, j);
-            PairNoise pn = pair_noise(seed, J >> 1, sig, tier, 0.0);
+            PairNoise pn = pair_noise(seed, J >> 1, sig, tier, 0.0, hp->antithetic ? -7 : -8);
             int code = load_code(w, t->bits, j);
-            w_out[i] = code + (int)applied_step(code, pn.delta[h], t->qmin, t->qmax, hp->boundary_mode);
+            w_out[i] = code + (int)applied_step(code, (long long)sign * pn.delta[h], t->qmin, t->qmax, hp->boundary_mode);
         }
     });
     return 0;

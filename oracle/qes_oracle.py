@@ -39,7 +39,8 @@ class _Tensor(C.Structure):
 
 class _HParams(C.Structure):
     _fields_ = [("sigma", C.c_float), ("lr", C.c_float), ("gamma", C.c_float),
-                ("n_pop", C.c_int32), ("sigma_unit", C.c_int32), ("boundary_mode", C.c_int32)]
+                ("n_pop", C.c_int32), ("sigma_unit", C.c_int32), ("boundary_mode", C.c_int32),
+                ("antithetic", C.c_int32)]
 
 
 @dataclass
@@ -70,9 +71,11 @@ class HParams:
     n_pop: int
     sigma_unit: int = 0      # 0 grid steps, 1 weight units (sigma / group scale)
     boundary_mode: int = 0   # 0 gate (Eq. 4), 1 clamp
+    antithetic: int = 0      # 1: n_pop / 2 seeded pairs (+delta, -delta); fitness interleaved F+, F-
 
     def c(self) -> _HParams:
-        return _HParams(self.sigma, self.lr, self.gamma, self.n_pop, self.sigma_unit, self.boundary_mode)
+        return _HParams(self.sigma, self.lr, self.gamma, self.n_pop, self.sigma_unit, self.boundary_mode,
+                        self.antithetic)
 
 
 _lib = None
@@ -128,13 +131,14 @@ def applied_step(w: int, step: int, qmin: int, qmax: int, mode: int) -> int:
     return lib().qo_applied_step(w, step, qmin, qmax, mode)
 
 
-def delta(seed: int, J, sigma_eff: float, tier: int = TIER_SPEC, tau: float = 0.0):
-    """Discrete perturbation of global elements J for one seed: (delta int32, x float64, near uint8)."""
+def delta(seed: int, J, sigma_eff: float, tier: int = TIER_SPEC, tau: float = 0.0, dmin: int = -8):
+    """Discrete perturbation of global elements J for one seed: (delta int32, x float64, near uint8).
+    dmin = -7 gives the symmetric 4-bit range used for antithetic pairs."""
     J = _arr(J, np.uint64)
     n = J.size
     d = np.empty(n, np.int32); x = np.empty(n, np.float64); near = np.empty(n, np.uint8)
     lib().qo_delta(C.c_uint64(seed), _p(J), C.c_int64(n), C.c_float(sigma_eff), C.c_int(tier),
-                   C.c_double(tau), _p(d), _p(x), _p(near))
+                   C.c_double(tau), C.c_int(dmin), _p(d), _p(x), _p(near))
     return d, x, near
 
 
@@ -174,11 +178,11 @@ def default_threads() -> int:
     return max(1, len(os.sched_getaffinity(0)))
 
 
-def perturb(t: Tensor, w, scales, seed: int, hp: HParams, tier=TIER_SPEC, idx=None, nthreads=None):
+def perturb(t: Tensor, w, scales, seed: int, hp: HParams, tier=TIER_SPEC, idx=None, nthreads=None, sign: int = 1):
     w = _arr(w, np.uint8); s = _scales(scales); idx, n = _idx(idx, t)
     out = np.empty(n, np.int32)
     tc, hc = t.c(), hp.c()
-    rc = lib().qo_perturb(C.byref(tc), _p(w), _p(s), C.c_uint64(seed), C.byref(hc), C.c_int(tier),
+    rc = lib().qo_perturb(C.byref(tc), _p(w), _p(s), C.c_uint64(seed), C.c_int(sign), C.byref(hc), C.c_int(tier),
                           _p(idx), C.c_int64(n), C.c_int(nthreads or default_threads()), _p(out))
     if rc:
         raise ValueError(f"oracle rejected arguments ({rc})")
@@ -195,7 +199,7 @@ def update(t: Tensor, w, scales, seeds, fitness, K: int, hp: HParams, residual_i
     """
     w = _arr(w, np.uint8); s = _scales(scales); idx, n = _idx(idx, t)
     seeds = _arr(seeds, np.uint64).reshape(-1); fitness = _arr(fitness, np.float32).reshape(-1)
-    assert seeds.size == (K + 1) * hp.n_pop and fitness.size == seeds.size
+    assert fitness.size == (K + 1) * hp.n_pop and seeds.size == fitness.size // (2 if hp.antithetic else 1)
     res = None if residual_in is None else _arr(residual_in, np.float32)
     out = dict(w_new=np.empty(n, np.int32), e_new=np.empty(n, np.float64), band=np.empty(n, np.float64),
                gate_final=np.empty(n, np.uint8), gate_replay=np.empty(n, np.int32),
@@ -215,7 +219,7 @@ def replay_residual(t: Tensor, w, scales, seeds, fitness, K: int, hp: HParams,
                     tier=TIER_SPEC, idx=None, nthreads=None):
     w = _arr(w, np.uint8); s = _scales(scales); idx, n = _idx(idx, t)
     seeds = _arr(seeds, np.uint64).reshape(-1); fitness = _arr(fitness, np.float32).reshape(-1)
-    assert seeds.size == K * hp.n_pop and fitness.size == seeds.size
+    assert fitness.size == K * hp.n_pop and seeds.size == fitness.size // (2 if hp.antithetic else 1)
     out = dict(e=np.empty(n, np.float64), band=np.empty(n, np.float64), gate_replay=np.empty(n, np.int32))
     tc, hc = t.c(), hp.c()
     rc = lib().qo_replay_residual(C.byref(tc), _p(w), _p(s), _p(seeds), _p(fitness), C.c_int(K),
