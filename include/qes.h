@@ -44,8 +44,8 @@ typedef enum {
     QES_ERR_BAD_BITS = -2,    /* bits is not 4 or 8 */
     QES_ERR_BAD_SHAPE = -3,   /* rows/cols/group_size/elem_offset violate the layout rules */
     QES_ERR_MISALIGNED = -4,  /* a device pointer misses its alignment (16 B weights/residual, 8 B seeds, 4 B fitness, 2 B scales) */
-    QES_ERR_BAD_HPARAM = -5,  /* sigma <= 0, n_pop <= 0, K < 0, gamma outside [0,1], qmin >= qmax, range outside the code width */
-    QES_ERR_BAD_MODE = -6,    /* unknown sigma_unit / boundary_mode, or residual_inout given with K > 0 */
+    QES_ERR_BAD_HPARAM = -5,  /* sigma <= 0, n_pop <= 0 (or odd with antithetic pairs), K < 0, gamma outside [0,1], qmin >= qmax, range outside the code width */
+    QES_ERR_BAD_MODE = -6,    /* unknown sigma_unit / boundary_mode / antithetic, residual_inout given with K > 0, qes_perturb_pair without antithetic, or its two outputs the same buffer */
     QES_ERR_CUDA = -7,        /* the launch reported a CUDA error (cudaGetLastError) */
     QES_ERR_TOO_LARGE = -8    /* n_pop exceeds what one generation's shared-memory staging holds (1066 members) */
 } qes_status;
@@ -68,6 +68,11 @@ typedef struct {
     int32_t n_pop;         /* population size N */
     int32_t sigma_unit;    /* QES_SIGMA_GRID | QES_SIGMA_WEIGHT */
     int32_t boundary_mode; /* QES_BOUNDARY_GATE | QES_BOUNDARY_CLAMP */
+    int32_t antithetic;    /* 0: N members, N seeds per generation.  1 (App. A, "antithetic perturbation
+                              pairs"): N even, N/2 pairs per generation, pair j = one seed and the two members
+                              W + delta_j, W - delta_j; seeds tables then hold N/2 entries per generation,
+                              fitness tables N entries per generation ordered F+_0, F-_0, F+_1, F-_1, ...,
+                              and delta is limited to the symmetric 4-bit range [-7, 7] */
 } qes_hparams;
 
 /*
@@ -75,15 +80,25 @@ typedef struct {
  *   w_in  [device, rows*cols codes]  current weights, not modified (unless w_out == w_in)
  *   w_out [device, same size]        perturbed weights; may alias w_in exactly, no partial overlap
  *   seed                             the member's seed s_i
- * Only sigma, sigma_unit and boundary_mode of hparams are used (n_pop, lr, gamma still validated).
+ * Only sigma, sigma_unit, boundary_mode and antithetic (which narrows delta to [-7, 7]) of hparams are
+ * used (n_pop, lr, gamma still validated).
  */
 int qes_perturb(const qes_tensor_desc* desc, const void* w_in, void* w_out, const void* scales_f16,
                 uint64_t seed, const qes_hparams* hparams, void* cuda_stream);
 
 /*
+ * Both members of one antithetic pair (App. A; Algorithm 1's member loop for members 2j and 2j+1) from a
+ * single evaluation of the noise: w_plus_out = Gate(W + delta), w_minus_out = Gate(W - delta), each gated
+ * (or clamped) on its own.  Requires hparams->antithetic == 1.  Either output may alias w_in exactly; the
+ * two outputs must be different, non-overlapping buffers.
+ */
+int qes_perturb_pair(const qes_tensor_desc* desc, const void* w_in, void* w_plus_out, void* w_minus_out,
+                     const void* scales_f16, uint64_t seed, const qes_hparams* hparams, void* cuda_stream);
+
+/*
  * Algorithm 2, history loop (proxy residual): for k = 0..K-1, u = alpha*g_k + gamma*e,
  * Delta = Round(u), gated against the CURRENT weights w, e = u - Delta_final.
- *   seeds   [device, K*n_pop uint64]  generation-major, oldest generation first
+ *   seeds   [device, K*n_pop uint64]  generation-major, oldest generation first (K*n_pop/2 with antithetic pairs)
  *   fitness [device, K*n_pop float]   same order
  *   residual_out [device, rows*cols float]  e after the K generations (K == 0 writes zeros)
  */
@@ -94,7 +109,8 @@ int qes_replay_residual(const qes_tensor_desc* desc, const void* w, const void* 
 /*
  * The update.  residual_inout == NULL: stateless (Algorithm 2) — replays K history generations
  * from e = 0, then applies the current generation; seeds/fitness hold K+1 generations, the last
- * row being the current one.  residual_inout != NULL: stored residual (Algorithm 1, Eqs. 6-8) —
+ * row being the current one (per generation n_pop seeds, or n_pop/2 with antithetic pairs, and
+ * n_pop fitness values).  residual_inout != NULL: stored residual (Algorithm 1, Eqs. 6-8) —
  * K must be 0; e is read, and e_{t+1} = u - Delta_final written back (fp32).
  *   w_inout [device]  updated in place: W <- W + Delta_final
  *   stats   [device, 4 x uint64, nullable]  counters ADDED to (caller zeroes): [0] codes changed,

@@ -30,7 +30,8 @@ class _TensorDesc(C.Structure):
 
 class _HParams(C.Structure):
     _fields_ = [("sigma", C.c_float), ("lr", C.c_float), ("gamma", C.c_float),
-                ("n_pop", C.c_int32), ("sigma_unit", C.c_int32), ("boundary_mode", C.c_int32)]
+                ("n_pop", C.c_int32), ("sigma_unit", C.c_int32), ("boundary_mode", C.c_int32),
+                ("antithetic", C.c_int32)]
 
 
 @dataclass
@@ -65,9 +66,15 @@ class HParams:
     n_pop: int
     sigma_unit: int = SIGMA_GRID
     boundary_mode: int = BOUNDARY_GATE
+    antithetic: int = 0
 
     def c(self) -> _HParams:
-        return _HParams(self.sigma, self.lr, self.gamma, self.n_pop, self.sigma_unit, self.boundary_mode)
+        return _HParams(self.sigma, self.lr, self.gamma, self.n_pop, self.sigma_unit, self.boundary_mode,
+                        self.antithetic)
+
+    @property
+    def seeds_per_generation(self) -> int:
+        return self.n_pop // 2 if self.antithetic else self.n_pop
 
 
 _lib = None
@@ -84,6 +91,8 @@ def load() -> C.CDLL:
         vp, u64, i32 = C.c_void_p, C.c_uint64, C.c_int32
         lib.qes_perturb.restype = C.c_int
         lib.qes_perturb.argtypes = [C.POINTER(_TensorDesc), vp, vp, vp, u64, C.POINTER(_HParams), vp]
+        lib.qes_perturb_pair.restype = C.c_int
+        lib.qes_perturb_pair.argtypes = [C.POINTER(_TensorDesc), vp, vp, vp, vp, u64, C.POINTER(_HParams), vp]
         lib.qes_replay_residual.restype = C.c_int
         lib.qes_replay_residual.argtypes = [C.POINTER(_TensorDesc), vp, vp, vp, vp, i32, C.POINTER(_HParams), vp, vp]
         lib.qes_update.restype = C.c_int
@@ -143,14 +152,26 @@ def qes_perturb(desc: TensorDesc, w_in, w_out, scales_f16, seed: int, hparams: H
     _check(rc)
 
 
+def qes_perturb_pair(desc: TensorDesc, w_in, w_plus_out, w_minus_out, scales_f16, seed: int, hparams: HParams,
+                     stream=None) -> None:
+    """Both members of one antithetic pair (App. A): Gate(W + delta) and Gate(W - delta) from one noise pass."""
+    d, h = desc.c(), hparams.c()
+    rc = load().qes_perturb_pair(C.byref(d), _ptr(w_in, dtype=_W, nbytes=desc.packed_bytes, name="w_in"),
+                                 _ptr(w_plus_out, dtype=_W, nbytes=desc.packed_bytes, name="w_plus_out"),
+                                 _ptr(w_minus_out, dtype=_W, nbytes=desc.packed_bytes, name="w_minus_out"),
+                                 _ptr(scales_f16, dtype=_S, nbytes=_scale_bytes(desc), name="scales"),
+                                 C.c_uint64(seed & 0xFFFFFFFFFFFFFFFF), C.byref(h), _stream(stream))
+    _check(rc)
+
+
 def qes_replay_residual(desc: TensorDesc, w, scales_f16, seeds, fitness, K: int, hparams: HParams,
                         residual_out, stream=None) -> None:
     """History loop of Algorithm 2: writes the proxy residual after K generations (fp32)."""
     d, h = desc.c(), hparams.c()
-    n = K * hparams.n_pop
+    n, ns = K * hparams.n_pop, K * hparams.seeds_per_generation
     rc = load().qes_replay_residual(C.byref(d), _ptr(w, dtype=_W, nbytes=desc.packed_bytes, name="w"),
                                     _ptr(scales_f16, dtype=_S, nbytes=_scale_bytes(desc), name="scales"),
-                                    _ptr(seeds, dtype=_SEEDS, nbytes=8 * n, name="seeds"),
+                                    _ptr(seeds, dtype=_SEEDS, nbytes=8 * ns, name="seeds"),
                                     _ptr(fitness, dtype=torch.float32, nbytes=4 * n, name="fitness"),
                                     K, C.byref(h),
                                     _ptr(residual_out, dtype=torch.float32, nbytes=4 * desc.numel, name="residual_out"),
@@ -162,10 +183,10 @@ def qes_update(desc: TensorDesc, w_inout, scales_f16, seeds, fitness, K: int, re
                hparams: HParams, stats=None, stream=None) -> None:
     """In-place update: stateless with seed replay (Algorithm 2) or with a stored residual (Algorithm 1)."""
     d, h = desc.c(), hparams.c()
-    n = (K + 1) * hparams.n_pop
+    n, ns = (K + 1) * hparams.n_pop, (K + 1) * hparams.seeds_per_generation
     rc = load().qes_update(C.byref(d), _ptr(w_inout, dtype=_W, nbytes=desc.packed_bytes, name="w_inout"),
                            _ptr(scales_f16, dtype=_S, nbytes=_scale_bytes(desc), name="scales"),
-                           _ptr(seeds, dtype=_SEEDS, nbytes=8 * n, name="seeds"),
+                           _ptr(seeds, dtype=_SEEDS, nbytes=8 * ns, name="seeds"),
                            _ptr(fitness, dtype=torch.float32, nbytes=4 * n, name="fitness"),
                            K, _ptr(residual_inout, dtype=torch.float32, nbytes=4 * desc.numel, name="residual_inout"),
                            C.byref(h), _ptr(stats, dtype=_SEEDS, nbytes=32, name="stats"), _stream(stream))

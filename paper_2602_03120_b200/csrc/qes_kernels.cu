@@ -36,6 +36,7 @@ constexpr int kSeedStride = 24;   // 32-bit words per staged member: a[10], b[10
 struct PassParams {
     const void* w_in;
     void* w_out;
+    void* w_out_minus;          // perturb only: the antithetic member W - delta (nullable)
     const unsigned short* scales;   // nullable, IEEE binary16 bits
     const uint64_t* seeds;
     const float* fitness;
@@ -46,7 +47,9 @@ struct PassParams {
     uint64_t elem_offset;
     int32_t group_size;
     int32_t generations;        // number of generations in the table
-    int32_t n_pop;
+    int32_t n_seeds;            // seeds per generation: n_pop, or n_pop / 2 antithetic pairs
+    int32_t antithetic;         // fitness holds 2 * n_seeds values per generation, F+ and F- interleaved
+    int32_t nd_max;             // largest -delta: 8, or 7 with antithetic pairs
     int32_t mode;               // PassMode
     int32_t boundary_mode;
     int32_t weight_unit;
@@ -85,9 +88,10 @@ __device__ __forceinline__ int applied_code(int w, int step, int qmin, int qmax,
     return min(max(target, qmin), qmax);
 }
 
-// Algorithm 1, member loop: W' = Gate(W + delta_i).  The member's round keys are computed on the
-// host and arrive as kernel parameters, i.e. as constant-bank operands.
-template <int BITS, bool CLAMP_DELTA>
+// Algorithm 1, member loop: W' = Gate(W + delta_i), and with PAIR also the antithetic member
+// Gate(W - delta_i) from the same noise.  The member's round keys are computed on the host and
+// arrive as kernel parameters, i.e. as constant-bank operands.
+template <int BITS, bool CLAMP_DELTA, bool PAIR>
 __global__ void __launch_bounds__(kThreads) perturb_kernel(PassParams p, RoundKeys rk) {
     int64_t chunk = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (chunk >= p.n_chunks) return;
@@ -97,28 +101,37 @@ __global__ void __launch_bounds__(kThreads) perturb_kernel(PassParams p, RoundKe
     uint64_t pair0 = (p.elem_offset >> 1) + (uint64_t)chunk * kPairs;
     uint32_t x0 = (uint32_t)pair0, y = (uint32_t)(pair0 >> 32);
     SeedConst sc = make_seed_const(y, rk);
-    Chunk<BITS, kPairs> out;
+    Chunk<BITS, kPairs> out, out_minus;
     out.clear();
+    out_minus.clear();
 #pragma unroll
     for (int i = 0; i < kPairs; ++i) {
         uint32_t r0, r1, r2, r3;
         philox_tail(make_pair_const(x0 + i), sc, rk, r0, r1, r2, r3);
         int z0, z1;
         pair_rounding_sums<CLAMP_DELTA>(r0, r1, r2, r3, nsig24, z0, z1);
+        int nd0 = neg_delta<CLAMP_DELTA>(z0, p.nd_max), nd1 = neg_delta<CLAMP_DELTA>(z1, p.nd_max);
         int w0 = w.get(2 * i), w1 = w.get(2 * i + 1);
-        out.put(2 * i, applied_code(w0, -neg_delta<CLAMP_DELTA>(z0), p.qmin_i, p.qmax_i, p.boundary_mode));
-        out.put(2 * i + 1, applied_code(w1, -neg_delta<CLAMP_DELTA>(z1), p.qmin_i, p.qmax_i, p.boundary_mode));
+        out.put(2 * i, applied_code(w0, -nd0, p.qmin_i, p.qmax_i, p.boundary_mode));
+        out.put(2 * i + 1, applied_code(w1, -nd1, p.qmin_i, p.qmax_i, p.boundary_mode));
+        if (PAIR) {
+            out_minus.put(2 * i, applied_code(w0, nd0, p.qmin_i, p.qmax_i, p.boundary_mode));
+            out_minus.put(2 * i + 1, applied_code(w1, nd1, p.qmin_i, p.qmax_i, p.boundary_mode));
+        }
     }
     out.store(p.w_out, chunk);
+    if (PAIR) out_minus.store(p.w_out_minus, chunk);
 }
 
 // Expands the seeds of one generation into round keys, next to the fitness values (stored as
 // -F * 2^-24, the factor that turns the kernel's -delta * 2^24 back into F * delta) and the
 // seed's SeedConst for counter high word y_cta (the one almost every CTA has throughout).
-__device__ __forceinline__ void stage_generation(uint32_t* buf, const uint64_t* seeds, const float* fitness, int n_pop,
-                                                 uint32_t y_cta) {
-    for (int i = threadIdx.x; i < n_pop; i += kThreads) {
+__device__ __noinline__ void stage_generation(uint32_t* buf, const uint64_t* seeds, const float* fitness, int n_seeds,
+                                                 bool antithetic, uint32_t y_cta) {
+    for (int i = threadIdx.x; i < n_seeds; i += kThreads) {
         uint64_t s = seeds[i];
+        // an antithetic pair contributes F+ * delta + F- * (-delta) to Eq. 5
+        float F = antithetic ? __fsub_rn(fitness[2 * i], fitness[2 * i + 1]) : fitness[i];
         RoundKeys rk = make_round_keys((uint32_t)s, (uint32_t)(s >> 32));
         SeedConst sc = make_seed_const(y_cta, rk);
         uint4* d = reinterpret_cast<uint4*>(buf + i * kSeedStride);
@@ -127,7 +140,7 @@ __device__ __forceinline__ void stage_generation(uint32_t* buf, const uint64_t* 
         d[2] = make_uint4(rk.a[8], rk.a[9], rk.b[0], rk.b[1]);
         d[3] = make_uint4(rk.b[2], rk.b[3], rk.b[4], rk.b[5]);
         d[4] = make_uint4(rk.b[6], rk.b[7], rk.b[8], rk.b[9]);
-        d[5] = make_uint4(__float_as_uint(fitness[i] * -0x1p-24f), sc.hak, sc.la, sc.lak);   // pairs with -delta * 2^24
+        d[5] = make_uint4(__float_as_uint(F * -0x1p-24f), sc.hak, sc.la, sc.lak);   // pairs with -delta * 2^24
     }
 }
 
@@ -181,7 +194,8 @@ __global__ void __launch_bounds__(kThreads, QES_MIN_BLOCKS) pass_kernel(PassPara
     }
 
     const int last = p.generations - 1;
-    const int buf_words = p.n_pop * kSeedStride;
+    const int buf_words = p.n_seeds * kSeedStride;
+    const int fit_per_gen = p.antithetic ? 2 * p.n_seeds : p.n_seeds;
     unsigned int n_changed = 0, n_blocked_final = 0, n_blocked_replay = 0, n_attempted = 0;
     Chunk<BITS, kPairs> out;
     out.clear();
@@ -192,19 +206,19 @@ __global__ void __launch_bounds__(kThreads, QES_MIN_BLOCKS) pass_kernel(PassPara
     const uint32_t y_cta = (uint32_t)(cta_pair0 >> 32);
     const bool y_uniform = (uint32_t)((cta_pair0 + (uint64_t)(kThreads * kPairs - 1)) >> 32) == y_cta;
 
-    if (p.generations > 0) stage_generation(smem, p.seeds, p.fitness, p.n_pop, y_cta);
+    if (p.generations > 0) stage_generation(smem, p.seeds, p.fitness, p.n_seeds, p.antithetic != 0, y_cta);
     for (int k = 0; k < p.generations; ++k) {
         __syncthreads();   // generation k is staged; nobody still reads the other buffer
         if (k < last)
-            stage_generation(smem + ((k + 1) & 1) * buf_words, p.seeds + (int64_t)(k + 1) * p.n_pop,
-                             p.fitness + (int64_t)(k + 1) * p.n_pop, p.n_pop, y_cta);
+            stage_generation(smem + ((k + 1) & 1) * buf_words, p.seeds + (int64_t)(k + 1) * p.n_seeds,
+                             p.fitness + (int64_t)(k + 1) * fit_per_gen, p.n_seeds, p.antithetic != 0, y_cta);
         if (!active) continue;
         const uint32_t* table = smem + (k & 1) * buf_words;
         float S[T];
 #pragma unroll
         for (int t = 0; t < T; ++t) S[t] = 0.0f;
 #pragma unroll 1
-        for (int i = 0; i < p.n_pop; ++i) {
+        for (int i = 0; i < p.n_seeds; ++i) {
             float Fm;   // -F_i * 2^-24
             SeedConst sc;
             const RoundKeys rk = load_round_keys(table + i * kSeedStride, Fm, sc);
@@ -215,8 +229,8 @@ __global__ void __launch_bounds__(kThreads, QES_MIN_BLOCKS) pass_kernel(PassPara
                 philox_tail(pc[pr], sc, rk, r0, r1, r2, r3);
                 int z0, z1;
                 pair_rounding_sums<CLAMP_DELTA>(r0, r1, r2, r3, nsig24, z0, z1);
-                S[2 * pr] = fmaf(Fm, neg_delta_scaled<CLAMP_DELTA>(z0), S[2 * pr]);            // Eq. 5 numerator
-                S[2 * pr + 1] = fmaf(Fm, neg_delta_scaled<CLAMP_DELTA>(z1), S[2 * pr + 1]);
+                S[2 * pr] = fmaf(Fm, neg_delta_scaled<CLAMP_DELTA>(z0, p.nd_max), S[2 * pr]);            // Eq. 5 numerator
+                S[2 * pr + 1] = fmaf(Fm, neg_delta_scaled<CLAMP_DELTA>(z1, p.nd_max), S[2 * pr + 1]);
             }
         }
         const bool is_update = (k == last) && (p.mode != kReplayOnly);
@@ -293,6 +307,8 @@ int validate(const qes_tensor_desc* d, const qes_hparams* h) {
     const int lo = -(1 << (d->bits - 1)), hi = (1 << (d->bits - 1)) - 1;
     if (d->qmin >= d->qmax || d->qmin < lo || d->qmax > hi) return QES_ERR_BAD_HPARAM;
     if (!(h->sigma > 0.0f) || !(h->sigma < 1e30f) || h->n_pop <= 0) return QES_ERR_BAD_HPARAM;
+    if (h->antithetic != 0 && h->antithetic != 1) return QES_ERR_BAD_MODE;
+    if (h->antithetic && (h->n_pop & 1)) return QES_ERR_BAD_HPARAM;
     if (!(h->gamma >= 0.0f && h->gamma <= 1.0f) || !(h->lr == h->lr)) return QES_ERR_BAD_HPARAM;
     if (h->sigma_unit != QES_SIGMA_GRID && h->sigma_unit != QES_SIGMA_WEIGHT) return QES_ERR_BAD_MODE;
     if (h->boundary_mode != QES_BOUNDARY_GATE && h->boundary_mode != QES_BOUNDARY_CLAMP) return QES_ERR_BAD_MODE;
@@ -306,7 +322,9 @@ PassParams base_params(const qes_tensor_desc* d, const qes_hparams* h, const voi
     p.cols = d->cols;
     p.elem_offset = d->elem_offset;
     p.group_size = d->group_size;
-    p.n_pop = h->n_pop;
+    p.n_seeds = h->antithetic ? h->n_pop / 2 : h->n_pop;
+    p.antithetic = h->antithetic;
+    p.nd_max = h->antithetic ? 7 : 8;
     p.boundary_mode = h->boundary_mode;
     p.weight_unit = h->sigma_unit == QES_SIGMA_WEIGHT;
     p.sigma = h->sigma;
@@ -325,11 +343,11 @@ bool delta_clamp_needed(const qes_hparams* h) {
     return h->sigma * 5.7682f + 1.0f > 7.0f;
 }
 
-size_t stage_bytes(int n_pop) { return (size_t)2 * (size_t)n_pop * kSeedStride * sizeof(uint32_t); }
+size_t stage_bytes(int n_seeds) { return (size_t)2 * (size_t)n_seeds * kSeedStride * sizeof(uint32_t); }
 
 template <int BITS, bool CLAMP, bool STATS>
 int launch_pass(const PassParams& p, cudaStream_t stream) {
-    const size_t smem = stage_bytes(p.n_pop);
+    const size_t smem = stage_bytes(p.n_seeds);
     if (smem > 48 * 1024) {
         cudaError_t a = cudaFuncSetAttribute(pass_kernel<BITS, CLAMP, STATS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (a != cudaSuccess) { cudaGetLastError(); return QES_ERR_CUDA; }
@@ -350,13 +368,51 @@ int dispatch_pass(int bits, bool clamp, const PassParams& p, cudaStream_t stream
     return bits == 4 ? dispatch_flags<4>(clamp, stats, p, stream) : dispatch_flags<8>(clamp, stats, p, stream);
 }
 
-int check_table(const uint64_t* seeds, const float* fitness, int64_t generations, int n_pop) {
+int check_table(const uint64_t* seeds, const float* fitness, int64_t generations, const qes_hparams* h) {
+    const int n_seeds = h->antithetic ? h->n_pop / 2 : h->n_pop;
     if (generations > 0) {
         if (seeds == nullptr || fitness == nullptr) return QES_ERR_NULL_PTR;
         if (!aligned(seeds, 8) || !aligned(fitness, 4)) return QES_ERR_MISALIGNED;
     }
-    if (stage_bytes(n_pop) > kMaxStageBytes) return QES_ERR_TOO_LARGE;
+    if (stage_bytes(n_seeds) > kMaxStageBytes) return QES_ERR_TOO_LARGE;
     return QES_OK;
+}
+
+template <int BITS>
+void launch_perturb_bits(bool clamp, bool pair, const PassParams& p, const RoundKeys& rk, unsigned blocks, cudaStream_t stream) {
+    if (clamp) {
+        if (pair) perturb_kernel<BITS, true, true><<<blocks, kThreads, 0, stream>>>(p, rk);
+        else perturb_kernel<BITS, true, false><<<blocks, kThreads, 0, stream>>>(p, rk);
+    } else {
+        if (pair) perturb_kernel<BITS, false, true><<<blocks, kThreads, 0, stream>>>(p, rk);
+        else perturb_kernel<BITS, false, false><<<blocks, kThreads, 0, stream>>>(p, rk);
+    }
+}
+
+// w_minus == nullptr: one member; otherwise both members of an antithetic pair.
+int launch_perturb(const qes_tensor_desc* desc, const void* w_in, void* w_out, void* w_minus, const void* scales_f16,
+                   uint64_t seed, const qes_hparams* hparams, void* cuda_stream) {
+    int rc = validate(desc, hparams);
+    if (rc != QES_OK) return rc;
+    if (w_in == nullptr || w_out == nullptr) return QES_ERR_NULL_PTR;
+    if (hparams->sigma_unit == QES_SIGMA_WEIGHT && scales_f16 == nullptr) return QES_ERR_NULL_PTR;
+    if (!aligned(w_in, 16) || !aligned(w_out, 16) || !aligned(w_minus, 16) || !aligned(scales_f16, 2)) return QES_ERR_MISALIGNED;
+    if (w_minus == w_out) return QES_ERR_BAD_MODE;
+    PassParams p = base_params(desc, hparams, scales_f16);
+    p.w_in = w_in;
+    p.w_out = w_out;
+    p.w_out_minus = w_minus;
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    unsigned blocks = (unsigned)((p.n_chunks + kThreads - 1) / kThreads);
+    RoundKeys rk;
+    for (int r = 0; r < 10; ++r) {
+        rk.a[r] = (uint32_t)seed + kPhiloxW0 * (uint32_t)r;
+        rk.b[r] = (uint32_t)(seed >> 32) + kPhiloxW1 * (uint32_t)r;
+    }
+    const bool clamp = delta_clamp_needed(hparams);
+    if (desc->bits == 4) launch_perturb_bits<4>(clamp, w_minus != nullptr, p, rk, blocks, stream);
+    else launch_perturb_bits<8>(clamp, w_minus != nullptr, p, rk, blocks, stream);
+    return cudaGetLastError() == cudaSuccess ? QES_OK : QES_ERR_CUDA;
 }
 
 }  // namespace qes
@@ -367,30 +423,14 @@ extern "C" {
 
 int qes_perturb(const qes_tensor_desc* desc, const void* w_in, void* w_out, const void* scales_f16,
                 uint64_t seed, const qes_hparams* hparams, void* cuda_stream) {
-    int rc = validate(desc, hparams);
-    if (rc != QES_OK) return rc;
-    if (w_in == nullptr || w_out == nullptr) return QES_ERR_NULL_PTR;
-    if (hparams->sigma_unit == QES_SIGMA_WEIGHT && scales_f16 == nullptr) return QES_ERR_NULL_PTR;
-    if (!aligned(w_in, 16) || !aligned(w_out, 16) || !aligned(scales_f16, 2)) return QES_ERR_MISALIGNED;
-    PassParams p = base_params(desc, hparams, scales_f16);
-    p.w_in = w_in;
-    p.w_out = w_out;
-    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
-    unsigned blocks = (unsigned)((p.n_chunks + kThreads - 1) / kThreads);
-    RoundKeys rk;
-    for (int r = 0; r < 10; ++r) {
-        rk.a[r] = (uint32_t)seed + kPhiloxW0 * (uint32_t)r;
-        rk.b[r] = (uint32_t)(seed >> 32) + kPhiloxW1 * (uint32_t)r;
-    }
-    bool clamp = delta_clamp_needed(hparams);
-    if (desc->bits == 4) {
-        if (clamp) perturb_kernel<4, true><<<blocks, kThreads, 0, stream>>>(p, rk);
-        else perturb_kernel<4, false><<<blocks, kThreads, 0, stream>>>(p, rk);
-    } else {
-        if (clamp) perturb_kernel<8, true><<<blocks, kThreads, 0, stream>>>(p, rk);
-        else perturb_kernel<8, false><<<blocks, kThreads, 0, stream>>>(p, rk);
-    }
-    return cudaGetLastError() == cudaSuccess ? QES_OK : QES_ERR_CUDA;
+    return launch_perturb(desc, w_in, w_out, nullptr, scales_f16, seed, hparams, cuda_stream);
+}
+
+int qes_perturb_pair(const qes_tensor_desc* desc, const void* w_in, void* w_plus_out, void* w_minus_out,
+                     const void* scales_f16, uint64_t seed, const qes_hparams* hparams, void* cuda_stream) {
+    if (w_minus_out == nullptr) return QES_ERR_NULL_PTR;
+    if (hparams != nullptr && hparams->antithetic != 1) return QES_ERR_BAD_MODE;
+    return launch_perturb(desc, w_in, w_plus_out, w_minus_out, scales_f16, seed, hparams, cuda_stream);
 }
 
 int qes_replay_residual(const qes_tensor_desc* desc, const void* w, const void* scales_f16,
@@ -402,7 +442,7 @@ int qes_replay_residual(const qes_tensor_desc* desc, const void* w, const void* 
     if (w == nullptr || residual_out == nullptr) return QES_ERR_NULL_PTR;
     if (hparams->sigma_unit == QES_SIGMA_WEIGHT && scales_f16 == nullptr) return QES_ERR_NULL_PTR;
     if (!aligned(w, 16) || !aligned(residual_out, 16) || !aligned(scales_f16, 2)) return QES_ERR_MISALIGNED;
-    rc = check_table(seeds, fitness, K, hparams->n_pop);
+    rc = check_table(seeds, fitness, K, hparams);
     if (rc != QES_OK) return rc;
     PassParams p = base_params(desc, hparams, scales_f16);
     p.w_in = w;
@@ -426,7 +466,7 @@ int qes_update(const qes_tensor_desc* desc, void* w_inout, const void* scales_f1
     if (hparams->sigma_unit == QES_SIGMA_WEIGHT && scales_f16 == nullptr) return QES_ERR_NULL_PTR;
     if (!aligned(w_inout, 16) || !aligned(residual_inout, 16) || !aligned(scales_f16, 2) || !aligned(stats, 8))
         return QES_ERR_MISALIGNED;
-    rc = check_table(seeds, fitness, (int64_t)K + 1, hparams->n_pop);
+    rc = check_table(seeds, fitness, (int64_t)K + 1, hparams);
     if (rc != QES_OK) return rc;
     PassParams p = base_params(desc, hparams, scales_f16);
     p.w_in = w_inout;
@@ -461,13 +501,13 @@ const char* qes_strerror(int status) {
         case QES_ERR_BAD_SHAPE: return "rows/cols/group_size/elem_offset violate the layout rules";
         case QES_ERR_MISALIGNED: return "a device pointer is not aligned as required";
         case QES_ERR_BAD_HPARAM: return "hyper-parameter or code range out of bounds";
-        case QES_ERR_BAD_MODE: return "unknown mode, or stored residual combined with K > 0";
+        case QES_ERR_BAD_MODE: return "unknown mode, stored residual combined with K > 0, or a pair call without antithetic set";
         case QES_ERR_CUDA: return "CUDA reported an error at launch";
         case QES_ERR_TOO_LARGE: return "n_pop exceeds the shared-memory staging limit";
         default: return "unknown status";
     }
 }
 
-int qes_version(void) { return 110; }
+int qes_version(void) { return 120; }
 
 }  // extern "C"

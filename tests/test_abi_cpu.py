@@ -19,7 +19,7 @@ def lib():
 def test_every_declared_symbol_is_exported(lib):
     header = open(os.path.join(ROOT, "include", "qes.h")).read()
     names = re.findall(r"^(?:int|const char\*)\s+(qes_\w+)\s*\(", header, flags=re.M)
-    assert set(names) >= {"qes_perturb", "qes_update", "qes_replay_residual", "qes_gaussian_factors", "qes_pipe_probe",
+    assert set(names) >= {"qes_perturb", "qes_update", "qes_replay_residual", "qes_perturb_pair", "qes_gaussian_factors", "qes_pipe_probe",
                           "qes_strerror", "qes_version"}
     for n in names:
         assert hasattr(lib, n), n
@@ -28,7 +28,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_struct_layouts_match_header():
     from paper_2602_03120_b200 import binding
-    assert C.sizeof(binding._TensorDesc) == 40 and C.sizeof(binding._HParams) == 24
+    assert C.sizeof(binding._TensorDesc) == 40 and C.sizeof(binding._HParams) == 28
     assert binding._TensorDesc.rows.offset == 16 and binding._TensorDesc.elem_offset.offset == 32
 
 
@@ -58,6 +58,15 @@ def test_invalid_arguments_are_rejected_without_launching(lib):
     assert lib.qes_perturb(None, 0x1000, 0x1000, None, 1, C.byref(h), None) == -1
     assert lib.qes_replay_residual(C.byref(d), 0x1000, None, 0x2000, 0x3000, 2, C.byref(h), None, None) == -1
     assert lib.qes_replay_residual(C.byref(d), 0x1000, None, 0x2000, 0x3000, 2, C.byref(h), 0x4008, None) == -4
+    # antithetic pairs: flag must be 0 or 1, the population even, the pair call needs the flag and two outputs
+    ha = lambda **kw: binding.HParams(**{**dict(sigma=0.5, lr=1.0, gamma=0.9, n_pop=4, antithetic=1), **kw}).c()
+    h2, h3, h1 = ha(antithetic=2), ha(n_pop=3), ha()
+    assert lib.qes_update(C.byref(d), 0x1000, None, 0x2000, 0x3000, 1, None, C.byref(h2), None, None) == -6
+    assert lib.qes_update(C.byref(d), 0x1000, None, 0x2000, 0x3000, 1, None, C.byref(h3), None, None) == -5
+    assert lib.qes_perturb_pair(C.byref(d), 0x1000, 0x5000, 0x6000, None, 1, C.byref(h), None) == -6
+    assert lib.qes_perturb_pair(C.byref(d), 0x1000, 0x5000, 0x5000, None, 1, C.byref(h1), None) == -6
+    assert lib.qes_perturb_pair(C.byref(d), 0x1000, 0x5000, None, None, 1, C.byref(h1), None) == -1
+    assert lib.qes_perturb_pair(C.byref(d), 0x1000, 0x5000, 0x6008, None, 1, C.byref(h1), None) == -4
     for code in range(-8, 1):
         assert len(lib.qes_strerror(code)) > 1
 

@@ -308,3 +308,40 @@ def test_update_where_the_counter_high_word_changes(qo, qes, bits, off):
     wp = _dev(np.zeros_like(packed))
     qes.qes_perturb(tg, _dev(packed), wp, None, int(seeds[0, 0]), hg)
     assert np.array_equal(_host(wp), qo.pack(bits, qo.perturb(to, packed, None, int(seeds[0, 0]), ho)))
+
+
+@pytest.mark.parametrize("bits,rows,cols,N,K,sigma,mode,unit", [
+    (4, 45, 736, 8, 4, 0.5, 0, 0), (8, 17, 288, 6, 2, 0.5, 1, 0), (4, 9, 512, 4, 3, 2.0, 0, 0), (4, 11, 256, 10, 1, 0.012, 0, 1)])
+def test_antithetic_pairs_update_replay_and_perturb(qo, qes, bits, rows, cols, N, K, sigma, mode, unit):
+    """App. A's antithetic pairs: N / 2 seeds per generation, fitness interleaved F+, F-; update, history loop
+    and the two-member perturbation against the oracle (sigma = 2.0 reaches the symmetric 4-bit limit)."""
+    import torch
+    group = 128 if (bits == 4 and unit) else 0
+    to, tg, packed, scales = _case(qo, qes, bits, rows, cols, group=group, off=32 * 77)
+    lr = 2.0 * sigma if unit else 1.0          # weight units: a step of the order of sigma, c = 2 / N
+    kw = dict(sigma=sigma, lr=lr, gamma=0.9, n_pop=N, boundary_mode=mode, sigma_unit=unit, antithetic=1)
+    ho, hg = _hp(qo, qes, **kw)
+    sc_d = _dev(scales) if unit else None
+    sc_o = scales if unit else None
+    seeds, fit = wl.draw_seeds(K + 1, N // 2, stream=rows), wl.draw_fitness(K + 1, N, stream=rows)
+    w = _dev(packed)
+    qes.qes_update(tg, w, sc_d, _dev(seeds), _dev(fit), K, None, hg)
+    ref = qo.update(to, packed, sc_o, seeds, fit, K, ho)
+    _compare_update(qo, _host(w), bits, ref, "antithetic update")
+    assert (ref["w_new"] != qo.unpack(bits, packed, rows * cols)).any()
+    res = torch.empty(rows * cols, dtype=torch.float32, device="cuda")
+    qes.qes_replay_residual(tg, _dev(packed), sc_d, _dev(seeds[:K]), _dev(fit[:K]), K, hg, res)
+    rr = qo.replay_residual(to, packed, sc_o, seeds[:K], fit[:K], K, ho)
+    far = rr["band"] >= BAND
+    assert np.abs(_host(res).astype(np.float64) - rr["e"])[far].max(initial=0.0) <= TOL
+    seed = int(seeds[-1, 0])
+    wp, wm = _dev(np.zeros_like(packed)), _dev(np.zeros_like(packed))
+    qes.qes_perturb_pair(tg, _dev(packed), wp, wm, sc_d, seed, hg)
+    assert np.array_equal(_host(wp), qo.pack(bits, qo.perturb(to, packed, sc_o, seed, ho, sign=1)))
+    assert np.array_equal(_host(wm), qo.pack(bits, qo.perturb(to, packed, sc_o, seed, ho, sign=-1)))
+    one = _dev(np.zeros_like(packed))
+    qes.qes_perturb(tg, _dev(packed), one, sc_d, seed, hg)               # the + member alone
+    assert np.array_equal(_host(one), _host(wp))
+    inplace = _dev(packed)
+    qes.qes_perturb_pair(tg, inplace, inplace, wm, sc_d, seed, hg)       # the + output may alias the input
+    assert np.array_equal(_host(inplace), _host(wp))
