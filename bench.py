@@ -94,7 +94,7 @@ class ClockSampler:
                 "power_w_max": max(pw) if pw else None, "samples": len(clk), "reasons": reasons}
 
 
-def oracle_rate(cfg: wl.Workload, target_seconds: float = 15.0):
+def oracle_rate(cfg: wl.Workload, target_seconds: float = 15.0, antithetic: bool = False):
     """Times the CPU oracle (as it stands) on a bounded sample of the workload: whole 32-element words
     drawn from the first tensor of the set, one full step on them (the perturbation of every member,
     then the stateless update) at the configuration's N and K.  Returns a dict."""
@@ -103,15 +103,18 @@ def oracle_rate(cfg: wl.Workload, target_seconds: float = 15.0):
     threads = qo.default_threads()
     t = cfg.tensors[0]
     packed = wl.draw_codes(cfg, 0)
-    seeds, fit = wl.draw_seeds(cfg.K + 1, cfg.n_pop), wl.draw_fitness(cfg.K + 1, cfg.n_pop, cfg.reward_dist)
+    n_seeds = cfg.n_pop // 2 if antithetic else cfg.n_pop
+    seeds, fit = wl.draw_seeds(cfg.K + 1, n_seeds), wl.draw_fitness(cfg.K + 1, cfg.n_pop, cfg.reward_dist)
     to = qo.Tensor(bits=cfg.bits, rows=t.rows, cols=t.cols, group_size=cfg.group_size, elem_offset=t.elem_offset)
-    hp = qo.HParams(sigma=cfg.sigma, lr=cfg.lr, gamma=cfg.gamma, n_pop=cfg.n_pop)
-    per_elem = cfg.n_pop * (cfg.K + 1)
+    hp = qo.HParams(sigma=cfg.sigma, lr=cfg.lr, gamma=cfg.gamma, n_pop=cfg.n_pop, antithetic=int(antithetic))
+    per_elem = n_seeds * (cfg.K + 1)
 
     def one_step(idx):
         t0 = time.perf_counter()
         for s in seeds[-1]:                                           # Algorithm 1, member loop
             qo.perturb(to, packed, None, int(s), hp, idx=idx)
+            if antithetic:
+                qo.perturb(to, packed, None, int(s), hp, idx=idx, sign=-1)
         qo.update(to, packed, None, seeds, fit, cfg.K, hp, idx=idx)   # Algorithm 2
         return time.perf_counter() - t0
 
@@ -131,13 +134,13 @@ def run_reference(args, cfg):
     if rank != 0:
         return
     per_step = max(1.0, min(20.0, 150.0 / max(1, args.steps + args.warmup)))
-    rates = [oracle_rate(cfg, per_step) for _ in range(args.warmup + args.steps)][args.warmup:]
+    rates = [oracle_rate(cfg, per_step, args.antithetic) for _ in range(args.warmup + args.steps)][args.warmup:]
     tot_w = sum(r["elements"] for r in rates); tot_t = sum(r["seconds"] for r in rates)
     value = tot_w / tot_t
     line = {"impl": "reference", "metric": "weights_updated_per_s", "value": value, "unit": "weights/s",
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot_t / len(rates),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int4+f32" if cfg.bits == 4 else "int8+f32",
-            "data": "synthetic", "config": config_dict(cfg, args.gpus),
+            "data": "synthetic", "config": config_dict(cfg, args.gpus, args.antithetic),
             "noise_samples_per_s": value * cfg.n_pop * (cfg.K + 1),
             "cpu_baseline": {"value": value, "unit": "weights/s", "cores": rates[0]["cores"], "kind": "oracle",
                              "sample": f"{rates[0]['elements']} elements (32-element words of tensor 0) per step, "
@@ -146,8 +149,8 @@ def run_reference(args, cfg):
     print(json.dumps(line))
 
 
-def config_dict(cfg, n_gpus):
-    return {"workload": cfg.name, "bits": cfg.bits, "weights_per_gpu": cfg.numel, "tensors_per_gpu": len(cfg.tensors),
+def config_dict(cfg, n_gpus, antithetic=False):
+    return {"population": "antithetic pairs" if antithetic else "independent members", "workload": cfg.name, "bits": cfg.bits, "weights_per_gpu": cfg.numel, "tensors_per_gpu": len(cfg.tensors),
             "n_pop": cfg.n_pop, "K": cfg.K, "sigma": cfg.sigma, "lr": cfg.lr, "gamma": cfg.gamma,
             "sigma_unit": "grid", "boundary": "gate", "perturb_members_per_step": cfg.n_pop,
             "launches": "one library call per run of consecutive tensors, at most 2^28 codes each",
@@ -163,6 +166,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="decoder7b_int4", choices=list(wl.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--antithetic", action="store_true",
+                    help="the population is N/2 antithetic pairs (App. A): N/2 seeds per generation, both members of a "
+                         "pair perturbed from one noise pass")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -190,15 +196,24 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    model = ModelPass(cfg, rank=rank, world=world)
+    model = ModelPass(cfg, rank=rank, world=world, antithetic=args.antithetic)
+    n_seeds = cfg.n_pop // 2 if args.antithetic else cfg.n_pop
     host = torch.from_numpy(model.host_codes()).pin_memory()
     host_out = torch.empty_like(host).pin_memory()
     model.load(host)
-    seeds_h = torch.from_numpy(wl.draw_seeds(cfg.K + 1, cfg.n_pop).view(np.int64)).pin_memory()
+    seeds_h = torch.from_numpy(wl.draw_seeds(cfg.K + 1, n_seeds).view(np.int64)).pin_memory()
     fit_h = torch.from_numpy(wl.draw_fitness(cfg.K + 1, cfg.n_pop, cfg.reward_dist)).pin_memory()
     seeds, fit = seeds_h.cuda(), fit_h.cuda()
-    member_seeds = [int(s) for s in wl.draw_seeds(cfg.K + 1, cfg.n_pop)[-1]]
+    member_seeds = [int(s) for s in wl.draw_seeds(cfg.K + 1, n_seeds)[-1]]
     scratch = torch.empty_like(model.w)
+    scratch_minus = torch.empty_like(model.w) if args.antithetic else None
+
+    def perturb_all():
+        n = 0
+        for s in member_seeds:                                  # Algorithm 1, member loop
+            n += model.perturb_pair(scratch, scratch_minus, s) if args.antithetic else model.perturb_member(scratch, s)
+        return n
+
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if model.bytes < (512 << 20) else None
     stream = torch.cuda.current_stream()
     ev = lambda: torch.cuda.Event(enable_timing=True)
@@ -209,8 +224,7 @@ def main():
             flush.fill_(1)
         if timers is not None:
             a, b, c = ev(), ev(), ev(); a.record(stream)
-        for s in member_seeds:                                  # Algorithm 1, member loop
-            launches += model.perturb_member(scratch, s)
+        launches += perturb_all()
         if timers is not None:
             b.record(stream)
         n_upd = model.update(seeds, fit, cfg.K)                 # Algorithm 2
@@ -250,8 +264,7 @@ def main():
         for _ in range(e2e_steps):
             model.load(host)
             s_d, f_d = seeds_h.cuda(non_blocking=True), fit_h.cuda(non_blocking=True)
-            for s in member_seeds:
-                model.perturb_member(scratch, s)
+            perturb_all()
             model.update(s_d, f_d, cfg.K)
             host_out.copy_(model.w, non_blocking=True)
         b.record(stream)
@@ -270,7 +283,7 @@ def main():
 
     hbm_gbs, sm_mhz, peak_src = measured_peaks()
     G = cfg.K + 1
-    upd_ops_per_launch = alu_ops(model.numel, cfg.n_pop, G) * args.steps / n_upd_launches
+    upd_ops_per_launch = alu_ops(model.numel, n_seeds, G) * args.steps / n_upd_launches
     upd_s_per_launch = update_ms * 1e-3 / n_upd_launches
     alu_peak = SM_COUNT * LANES_PER_SM * sm_mhz * 1e6
     achieved = upd_ops_per_launch / upd_s_per_launch
@@ -287,13 +300,13 @@ def main():
     line = {"metric": "weights_updated_per_s", "value": value, "unit": "weights/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "int4+f32" if cfg.bits == 4 else "int8+f32",
-            "data": "synthetic", "config": config_dict(cfg, world),
-            "noise_samples_per_s": world * model.numel * cfg.n_pop * G / (update_ms * 1e-3 / args.steps),
+            "data": "synthetic", "config": config_dict(cfg, world, args.antithetic),
+            "noise_samples_per_s": world * model.numel * n_seeds * G / (update_ms * 1e-3 / args.steps),
             "update_ms_per_step": update_ms / args.steps, "perturb_ms_per_step": perturb_ms / args.steps,
             "perturb_weights_per_s": world * model.numel * cfg.n_pop / (perturb_ms * 1e-3 / args.steps),
             "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "e2e": e2e}
     if not args.no_cpu_baseline and world == 1:
-        r = oracle_rate(cfg)
+        r = oracle_rate(cfg, antithetic=args.antithetic)
         line["cpu_baseline"] = {"value": r["weights_per_s"], "unit": "weights/s", "cores": r["cores"], "kind": "oracle",
                                 "samples_per_s": r["samples_per_s"],
                                 "sample": f"{r['elements']} elements (32-element words of tensor 0), one full step (perturb x N, update), "

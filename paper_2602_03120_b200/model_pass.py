@@ -46,7 +46,8 @@ def launch_segments(tensors, max_elems: int = MAX_SEGMENT_ELEMS):
 
 class ModelPass:
     def __init__(self, workload: wl.Workload, device="cuda", rank: int = 0, world: int = 1,
-                 sigma_unit: int = qes.SIGMA_GRID, with_scales: bool = False, tensors=None):
+                 sigma_unit: int = qes.SIGMA_GRID, with_scales: bool = False, tensors=None,
+                 antithetic: bool = False):
         self.wl = workload
         self.device = torch.device(device)
         self.tensors = tuple(tensors) if tensors is not None else shard_tensors(workload, rank, world)
@@ -55,7 +56,7 @@ class ModelPass:
         self.bytes = wl.packed_bytes(workload.bits, self.numel)
         self.w = torch.empty(self.bytes, dtype=torch.uint8, device=self.device)
         self.hp = qes.HParams(sigma=workload.sigma, lr=workload.lr, gamma=workload.gamma, n_pop=workload.n_pop,
-                              sigma_unit=sigma_unit)
+                              sigma_unit=sigma_unit, antithetic=int(antithetic))
         self.descs = [qes.TensorDesc(bits=workload.bits, rows=t.rows, cols=t.cols, group_size=workload.group_size,
                                      elem_offset=t.elem_offset) for t in self.tensors]
         # grid-unit sigma: fused launches over runs of tensors; weight-unit sigma: one launch per tensor
@@ -97,6 +98,14 @@ class ModelPass:
         calls = self._launches()
         for t, d, sc in calls:
             qes.qes_perturb(d, self._slice(self.w, t), self._slice(out, t), sc, seed, self.hp)
+        return len(calls)
+
+    def perturb_pair(self, out_plus: torch.Tensor, out_minus: torch.Tensor, seed: int) -> int:
+        """Both members of one antithetic pair (App. A) from one noise pass."""
+        calls = self._launches()
+        for t, d, sc in calls:
+            qes.qes_perturb_pair(d, self._slice(self.w, t), self._slice(out_plus, t), self._slice(out_minus, t), sc,
+                                 seed, self.hp)
         return len(calls)
 
     def update(self, seeds: torch.Tensor, fitness: torch.Tensor, K: int, stats=None) -> int:
