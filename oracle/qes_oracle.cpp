@@ -174,6 +174,24 @@ float half_to_float(uint16_t h) {
     return u2f(sign | ((uint32_t)(exp + 112) << 23) | (man << 13));
 }
 
+// double -> IEEE binary16, round to nearest even, written out from the format's definition
+// (10 fraction bits, exponent bias 15, gradual underflow below 2^-14, overflow to infinity).
+uint16_t double_to_half(double v) {
+    uint16_t sign = std::signbit(v) ? 0x8000u : 0u;
+    double a = std::fabs(v);
+    if (std::isnan(v)) return (uint16_t)(sign | 0x7e00u);
+    if (a >= 65520.0) return (uint16_t)(sign | 0x7c00u);          // rounds to infinity
+    if (a < 0x1p-25) return sign;                                  // below half the smallest subnormal (ties to even: 0)
+    int ex;
+    std::frexp(a, &ex);                                            // a = m * 2^ex, m in [0.5, 1)
+    int e = std::max(ex - 1, -14);                                 // exponent of the binary16 grid at a
+    double scaled = std::ldexp(a, 10 - e);                         // in units of the grid spacing 2^(e-10)
+    double r = std::nearbyint(scaled);                             // default rounding mode: nearest even
+    if (r >= 2048.0) { r = 1024.0; e += 1; }                       // carried into the next binade
+    if (e == -14 && r < 1024.0) return (uint16_t)(sign | (uint16_t)r);              // subnormal
+    return (uint16_t)(sign | (uint16_t)((e + 15) << 10) | ((uint16_t)r & 0x3ffu));
+}
+
 // Row-major [rows, cols].  INT4: two codes per byte, even column in the low
 // nibble, two's complement.  INT8: one signed byte per code.
 int load_code(const uint8_t* packed, int bits, int64_t j) {
@@ -193,7 +211,9 @@ struct Tensor { int32_t bits, qmin, qmax, group_size; int64_t rows, cols; uint64
 // antithetic != 0 (App. A "antithetic perturbation pairs"): the population is n_pop / 2 pairs, pair j
 // has one seed and the two members W + delta_j and W - delta_j; seeds hold n_pop / 2 entries per
 // generation, fitness holds n_pop entries per generation ordered F+_0, F-_0, F+_1, F-_1, ...
-struct HParams { float sigma, lr, gamma; int32_t n_pop, sigma_unit, boundary_mode, antithetic; };
+// residual_f16 != 0: the stored residual of Algorithm 1 is kept in binary16 ("Residuals e_0 <- 0 (FP16)"):
+// read as binary16, all arithmetic as before; the caller rounds the returned e back to binary16.
+struct HParams { float sigma, lr, gamma; int32_t n_pop, sigma_unit, boundary_mode, antithetic, residual_f16; };
 
 float sigma_eff(const Tensor& t, const HParams& hp, const uint16_t* scales, int64_t j) {
     if (hp.sigma_unit == 0) return hp.sigma;                    // sigma in grid steps
@@ -306,6 +326,12 @@ int qo_stochastic_round(float x, uint32_t rword) { return stochastic_round_f32(x
 
 float qo_half_to_float(uint16_t h) { return half_to_float(h); }
 
+uint16_t qo_double_to_half(double v) { return double_to_half(v); }
+
+void qo_doubles_to_halves(const double* v, int64_t n, uint16_t* out) {
+    for (int64_t i = 0; i < n; ++i) out[i] = double_to_half(v[i]);
+}
+
 // delta (and optionally x = sigma_eff * eps, near-decision flags) of global
 // elements J[0..n) for one seed and one sigma_eff.
 void qo_delta(uint64_t seed, const uint64_t* J, int64_t n, float sigma_eff_v, int tier, double tau, int dmin,
@@ -360,7 +386,7 @@ int qo_perturb(const Tensor* t, const uint8_t* w, const uint16_t* scales, uint64
 // final step was blocked, number of blocked replay steps, whether the final
 // rounded step was non-zero.
 int qo_update(const Tensor* t, const uint8_t* w, const uint16_t* scales, const uint64_t* seeds,
-              const float* fitness, int K, const float* residual_in, const HParams* hp, int tier,
+              const float* fitness, int K, const void* residual_in, const HParams* hp, int tier,
               const int64_t* idx, int64_t n, int nthreads,
               int32_t* w_new, double* e_new, double* band, uint8_t* gate_final, int32_t* gate_replay,
               uint8_t* attempted) {
@@ -372,7 +398,10 @@ int qo_update(const Tensor* t, const uint8_t* w, const uint16_t* scales, const u
         for (int64_t i = lo; i < hi; ++i) {
             int64_t j = idx ? idx[i] : i;
             int code = load_code(w, t->bits, j);
-            double e0 = residual_in ? (double)residual_in[j] : 0.0;
+            double e0 = 0.0;
+            if (residual_in)
+                e0 = hp->residual_f16 ? (double)half_to_float(((const uint16_t*)residual_in)[j])
+                                      : (double)((const float*)residual_in)[j];
             ElemResult r = element_update(*t, *hp, scales, code, j, seeds, fitness, K + 1, e0, false, tier);
             w_new[i] = r.w_new;
             if (e_new) e_new[i] = r.e_new;

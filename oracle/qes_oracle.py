@@ -40,7 +40,7 @@ class _Tensor(C.Structure):
 class _HParams(C.Structure):
     _fields_ = [("sigma", C.c_float), ("lr", C.c_float), ("gamma", C.c_float),
                 ("n_pop", C.c_int32), ("sigma_unit", C.c_int32), ("boundary_mode", C.c_int32),
-                ("antithetic", C.c_int32)]
+                ("antithetic", C.c_int32), ("residual_f16", C.c_int32)]
 
 
 @dataclass
@@ -72,10 +72,11 @@ class HParams:
     sigma_unit: int = 0      # 0 grid steps, 1 weight units (sigma / group scale)
     boundary_mode: int = 0   # 0 gate (Eq. 4), 1 clamp
     antithetic: int = 0      # 1: n_pop / 2 seeded pairs (+delta, -delta); fitness interleaved F+, F-
+    residual_f16: int = 0    # 1: the stored residual is binary16
 
     def c(self) -> _HParams:
         return _HParams(self.sigma, self.lr, self.gamma, self.n_pop, self.sigma_unit, self.boundary_mode,
-                        self.antithetic)
+                        self.antithetic, self.residual_f16)
 
 
 _lib = None
@@ -89,6 +90,8 @@ def lib() -> C.CDLL:
         _lib.qo_half_to_float.argtypes = [C.c_uint16]
         _lib.qo_stochastic_round.restype = C.c_int
         _lib.qo_stochastic_round.argtypes = [C.c_float, C.c_uint32]
+        _lib.qo_double_to_half.restype = C.c_uint16
+        _lib.qo_double_to_half.argtypes = [C.c_double]
         _lib.qo_applied_step.restype = C.c_longlong
         _lib.qo_applied_step.argtypes = [C.c_int, C.c_longlong, C.c_int, C.c_int, C.c_int]
     return _lib
@@ -125,6 +128,14 @@ def stochastic_round(x: float, rword: int) -> int:
 
 def half_to_float(h: int) -> float:
     return lib().qo_half_to_float(C.c_uint16(h))
+
+
+def to_half(values) -> np.ndarray:
+    """Rounds doubles to binary16 (nearest even); returns the bit patterns as uint16."""
+    v = _arr(values, np.float64).reshape(-1)
+    out = np.empty(v.size, np.uint16)
+    lib().qo_doubles_to_halves(_p(v), C.c_int64(v.size), _p(out))
+    return out
 
 
 def applied_step(w: int, step: int, qmin: int, qmax: int, mode: int) -> int:
@@ -200,7 +211,14 @@ def update(t: Tensor, w, scales, seeds, fitness, K: int, hp: HParams, residual_i
     w = _arr(w, np.uint8); s = _scales(scales); idx, n = _idx(idx, t)
     seeds = _arr(seeds, np.uint64).reshape(-1); fitness = _arr(fitness, np.float32).reshape(-1)
     assert fitness.size == (K + 1) * hp.n_pop and seeds.size == fitness.size // (2 if hp.antithetic else 1)
-    res = None if residual_in is None else _arr(residual_in, np.float32)
+    if residual_in is None:
+        res = None
+    elif hp.residual_f16:
+        res = np.ascontiguousarray(residual_in)
+        res = res.view(np.uint16) if res.dtype == np.float16 else res
+        assert res.dtype == np.uint16
+    else:
+        res = _arr(residual_in, np.float32)
     out = dict(w_new=np.empty(n, np.int32), e_new=np.empty(n, np.float64), band=np.empty(n, np.float64),
                gate_final=np.empty(n, np.uint8), gate_replay=np.empty(n, np.int32),
                attempted=np.empty(n, np.uint8))

@@ -45,3 +45,20 @@ def test_gate_and_clamp_exhaustive(qo):
                 assert w + c == min(qmax, max(qmin, w + step))  # saturating variant
                 if inside:
                     assert g == c == step
+
+
+def test_half_encode_matches_numpy_and_roundtrips(qo):
+    """binary16 rounding (nearest even) on every representable value, every midpoint between neighbours,
+    random doubles over the whole range, subnormals, overflow and signed zero."""
+    all_bits = np.arange(1 << 16, dtype=np.uint16)
+    vals = all_bits.view(np.float16).astype(np.float64)
+    finite = np.isfinite(vals)
+    assert np.array_equal(qo.to_half(vals[finite]), all_bits[finite])            # round trip
+    pos = np.sort(vals[finite & (vals >= 0)])
+    mids = (pos[:-1] + pos[1:]) / 2.0                                            # ties go to the even neighbour
+    rng = np.random.default_rng(0)
+    rnd = np.concatenate([rng.standard_normal(200_000) * 10.0 ** rng.integers(-9, 5, 200_000), mids, -mids,
+                          [65519.9, 65520.0, 1e9, -1e9, 2.0 ** -25, 2.0 ** -25 * 1.0000001, 0.0, -0.0]])
+    with np.errstate(over="ignore"):
+        want = rnd.astype(np.float16).view(np.uint16)
+    assert np.array_equal(qo.to_half(rnd), want)
