@@ -73,6 +73,9 @@ typedef struct {
                               W + delta_j, W - delta_j; seeds tables then hold N/2 entries per generation,
                               fitness tables N entries per generation ordered F+_0, F-_0, F+_1, F-_1, ...,
                               and delta is limited to the symmetric 4-bit range [-7, 7] */
+    int32_t residual_f16;  /* format of residual_inout / residual_out: 0 = float, 1 = IEEE binary16 (Algorithm 1,
+                              "Residuals e_0 <- 0 (FP16)"): read as binary16, arithmetic in fp32, rounded to
+                              nearest even on the store */
 } qes_hparams;
 
 /*
@@ -100,25 +103,27 @@ int qes_perturb_pair(const qes_tensor_desc* desc, const void* w_in, void* w_plus
  * Delta = Round(u), gated against the CURRENT weights w, e = u - Delta_final.
  *   seeds   [device, K*n_pop uint64]  generation-major, oldest generation first (K*n_pop/2 with antithetic pairs)
  *   fitness [device, K*n_pop float]   same order
- *   residual_out [device, rows*cols float]  e after the K generations (K == 0 writes zeros)
+ *   residual_out [device, rows*cols float, or binary16 with hparams->residual_f16; 16-byte aligned]
+ *                e after the K generations (K == 0 writes zeros)
  */
 int qes_replay_residual(const qes_tensor_desc* desc, const void* w, const void* scales_f16,
                         const uint64_t* seeds, const float* fitness, int32_t K,
-                        const qes_hparams* hparams, float* residual_out, void* cuda_stream);
+                        const qes_hparams* hparams, void* residual_out, void* cuda_stream);
 
 /*
  * The update.  residual_inout == NULL: stateless (Algorithm 2) — replays K history generations
  * from e = 0, then applies the current generation; seeds/fitness hold K+1 generations, the last
  * row being the current one (per generation n_pop seeds, or n_pop/2 with antithetic pairs, and
  * n_pop fitness values).  residual_inout != NULL: stored residual (Algorithm 1, Eqs. 6-8) —
- * K must be 0; e is read, and e_{t+1} = u - Delta_final written back (fp32).
+ * K must be 0; e is read, and e_{t+1} = u - Delta_final written back (float, or binary16 with
+ * hparams->residual_f16; rows*cols elements, 16-byte aligned).
  *   w_inout [device]  updated in place: W <- W + Delta_final
  *   stats   [device, 4 x uint64, nullable]  counters ADDED to (caller zeroes): [0] codes changed,
  *           [1] final steps blocked or shortened by the boundary, [2] blocked replay steps,
  *           [3] non-zero rounded final steps (before the boundary rule)
  */
 int qes_update(const qes_tensor_desc* desc, void* w_inout, const void* scales_f16,
-               const uint64_t* seeds, const float* fitness, int32_t K, float* residual_inout,
+               const uint64_t* seeds, const float* fitness, int32_t K, void* residual_inout,
                const qes_hparams* hparams, uint64_t* stats, void* cuda_stream);
 
 /*

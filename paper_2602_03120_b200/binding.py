@@ -31,7 +31,7 @@ class _TensorDesc(C.Structure):
 class _HParams(C.Structure):
     _fields_ = [("sigma", C.c_float), ("lr", C.c_float), ("gamma", C.c_float),
                 ("n_pop", C.c_int32), ("sigma_unit", C.c_int32), ("boundary_mode", C.c_int32),
-                ("antithetic", C.c_int32)]
+                ("antithetic", C.c_int32), ("residual_f16", C.c_int32)]
 
 
 @dataclass
@@ -67,10 +67,19 @@ class HParams:
     sigma_unit: int = SIGMA_GRID
     boundary_mode: int = BOUNDARY_GATE
     antithetic: int = 0
+    residual_f16: int = 0
 
     def c(self) -> _HParams:
         return _HParams(self.sigma, self.lr, self.gamma, self.n_pop, self.sigma_unit, self.boundary_mode,
-                        self.antithetic)
+                        self.antithetic, self.residual_f16)
+
+    @property
+    def residual_dtype(self):
+        return torch.float16 if self.residual_f16 else torch.float32
+
+    @property
+    def residual_itemsize(self) -> int:
+        return 2 if self.residual_f16 else 4
 
     @property
     def seeds_per_generation(self) -> int:
@@ -174,7 +183,8 @@ def qes_replay_residual(desc: TensorDesc, w, scales_f16, seeds, fitness, K: int,
                                     _ptr(seeds, dtype=_SEEDS, nbytes=8 * ns, name="seeds"),
                                     _ptr(fitness, dtype=torch.float32, nbytes=4 * n, name="fitness"),
                                     K, C.byref(h),
-                                    _ptr(residual_out, dtype=torch.float32, nbytes=4 * desc.numel, name="residual_out"),
+                                    _ptr(residual_out, dtype=hparams.residual_dtype, nbytes=hparams.residual_itemsize * desc.numel,
+                                         name="residual_out"),
                                     _stream(stream))
     _check(rc)
 
@@ -188,7 +198,8 @@ def qes_update(desc: TensorDesc, w_inout, scales_f16, seeds, fitness, K: int, re
                            _ptr(scales_f16, dtype=_S, nbytes=_scale_bytes(desc), name="scales"),
                            _ptr(seeds, dtype=_SEEDS, nbytes=8 * ns, name="seeds"),
                            _ptr(fitness, dtype=torch.float32, nbytes=4 * n, name="fitness"),
-                           K, _ptr(residual_inout, dtype=torch.float32, nbytes=4 * desc.numel, name="residual_inout"),
+                           K, _ptr(residual_inout, dtype=hparams.residual_dtype,
+                                   nbytes=hparams.residual_itemsize * desc.numel, name="residual_inout"),
                            C.byref(h), _ptr(stats, dtype=_SEEDS, nbytes=32, name="stats"), _stream(stream))
     _check(rc)
 

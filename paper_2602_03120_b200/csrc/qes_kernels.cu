@@ -40,7 +40,8 @@ struct PassParams {
     const unsigned short* scales;   // nullable, IEEE binary16 bits
     const uint64_t* seeds;
     const float* fitness;
-    float* residual;            // stored-residual in/out, or replay output
+    void* residual;             // stored-residual in/out, or replay output: fp32, or binary16 when residual_f16
+    int32_t residual_f16;
     unsigned long long* stats;  // nullable
     int64_t n_chunks;
     int64_t cols;
@@ -72,6 +73,55 @@ __device__ __forceinline__ float chunk_neg_sigma24(const PassParams& p, int64_t 
     int64_t row = j / p.cols;
     int64_t g = p.group_size > 0 ? row * (p.cols / p.group_size) + (j - row * p.cols) / p.group_size : row;
     return -fminf(__fdiv_rn(p.sigma, half_bits_to_float(p.scales[g])), 0x1p40f) * 0x1p24f;
+}
+
+// The T residuals of one thread, fp32 or binary16 (Algorithm 1 keeps e in FP16), as 128-bit accesses.
+template <int T>
+__device__ __forceinline__ void load_residual(const void* base, bool f16, int64_t chunk, float (&e)[T]) {
+    static_assert(T % 8 == 0, "a thread owns a multiple of eight residuals");
+    if (f16) {
+        const uint4* r = reinterpret_cast<const uint4*>(base) + chunk * (T / 8);
+#pragma unroll
+        for (int q = 0; q < T / 8; ++q) {
+            uint4 v = r[q];
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                e[8 * q + 2 * i] = half_bits_to_float((unsigned short)(w[i] & 0xffffu));
+                e[8 * q + 2 * i + 1] = half_bits_to_float((unsigned short)(w[i] >> 16));
+            }
+        }
+    } else {
+        const float4* r4 = reinterpret_cast<const float4*>(base) + chunk * (T / 4);
+#pragma unroll
+        for (int q = 0; q < T / 4; ++q) {
+            float4 v = r4[q];
+            e[4 * q] = v.x; e[4 * q + 1] = v.y; e[4 * q + 2] = v.z; e[4 * q + 3] = v.w;
+        }
+    }
+}
+
+__device__ __forceinline__ uint32_t float_to_half_bits(float x) {
+    return (uint32_t)__half_as_ushort(__float2half_rn(x));
+}
+
+template <int T>
+__device__ __forceinline__ void store_residual(void* base, bool f16, int64_t chunk, const float (&e)[T]) {
+    if (f16) {
+        uint4* r = reinterpret_cast<uint4*>(base) + chunk * (T / 8);
+#pragma unroll
+        for (int q = 0; q < T / 8; ++q) {
+            uint32_t w[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                w[i] = float_to_half_bits(e[8 * q + 2 * i]) | (float_to_half_bits(e[8 * q + 2 * i + 1]) << 16);
+            r[q] = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+    } else {
+        float4* r4 = reinterpret_cast<float4*>(base) + chunk * (T / 4);
+#pragma unroll
+        for (int q = 0; q < T / 4; ++q) r4[q] = make_float4(e[4 * q], e[4 * q + 1], e[4 * q + 2], e[4 * q + 3]);
+    }
 }
 
 // Eq. 4 (gate) or saturation: the step actually applied to code w for a rounded step.
@@ -177,14 +227,7 @@ __global__ void __launch_bounds__(kThreads, QES_MIN_BLOCKS) pass_kernel(PassPara
     uint32_t y = 0u;
     if (active) {
         w.load(p.w_in, chunk);
-        if (p.mode == kStoredResidual) {
-            const float4* r4 = reinterpret_cast<const float4*>(p.residual) + chunk * (T / 4);
-#pragma unroll
-            for (int q = 0; q < T / 4; ++q) {
-                float4 v = r4[q];
-                e[4 * q] = v.x; e[4 * q + 1] = v.y; e[4 * q + 2] = v.z; e[4 * q + 3] = v.w;
-            }
-        }
+        if (p.mode == kStoredResidual) load_residual<T>(p.residual, p.residual_f16 != 0, chunk, e);
         nsig24 = chunk_neg_sigma24(p, chunk);
         // a thread's pairs share the counter high word: pair0 is a multiple of kPairs
         const uint64_t pair0 = (p.elem_offset >> 1) + (uint64_t)chunk * kPairs;
@@ -257,11 +300,7 @@ __global__ void __launch_bounds__(kThreads, QES_MIN_BLOCKS) pass_kernel(PassPara
 
     if (active) {
         if (p.mode != kReplayOnly) out.store(p.w_out, chunk);
-        if (p.mode != kStateless) {
-            float4* r4 = reinterpret_cast<float4*>(p.residual) + chunk * (T / 4);
-#pragma unroll
-            for (int q = 0; q < T / 4; ++q) r4[q] = make_float4(e[4 * q], e[4 * q + 1], e[4 * q + 2], e[4 * q + 3]);
-        }
+        if (p.mode != kStateless) store_residual<T>(p.residual, p.residual_f16 != 0, chunk, e);
     }
     if (STATS) {
         // inactive threads carry zeros: every warp of the CTA is whole here
@@ -308,6 +347,7 @@ int validate(const qes_tensor_desc* d, const qes_hparams* h) {
     if (d->qmin >= d->qmax || d->qmin < lo || d->qmax > hi) return QES_ERR_BAD_HPARAM;
     if (!(h->sigma > 0.0f) || !(h->sigma < 1e30f) || h->n_pop <= 0) return QES_ERR_BAD_HPARAM;
     if (h->antithetic != 0 && h->antithetic != 1) return QES_ERR_BAD_MODE;
+    if (h->residual_f16 != 0 && h->residual_f16 != 1) return QES_ERR_BAD_MODE;
     if (h->antithetic && (h->n_pop & 1)) return QES_ERR_BAD_HPARAM;
     if (!(h->gamma >= 0.0f && h->gamma <= 1.0f) || !(h->lr == h->lr)) return QES_ERR_BAD_HPARAM;
     if (h->sigma_unit != QES_SIGMA_GRID && h->sigma_unit != QES_SIGMA_WEIGHT) return QES_ERR_BAD_MODE;
@@ -324,6 +364,7 @@ PassParams base_params(const qes_tensor_desc* d, const qes_hparams* h, const voi
     p.group_size = d->group_size;
     p.n_seeds = h->antithetic ? h->n_pop / 2 : h->n_pop;
     p.antithetic = h->antithetic;
+    p.residual_f16 = h->residual_f16;
     p.nd_max = h->antithetic ? 7 : 8;
     p.boundary_mode = h->boundary_mode;
     p.weight_unit = h->sigma_unit == QES_SIGMA_WEIGHT;
@@ -435,7 +476,7 @@ int qes_perturb_pair(const qes_tensor_desc* desc, const void* w_in, void* w_plus
 
 int qes_replay_residual(const qes_tensor_desc* desc, const void* w, const void* scales_f16,
                         const uint64_t* seeds, const float* fitness, int32_t K,
-                        const qes_hparams* hparams, float* residual_out, void* cuda_stream) {
+                        const qes_hparams* hparams, void* residual_out, void* cuda_stream) {
     int rc = validate(desc, hparams);
     if (rc != QES_OK) return rc;
     if (K < 0) return QES_ERR_BAD_HPARAM;
@@ -456,7 +497,7 @@ int qes_replay_residual(const qes_tensor_desc* desc, const void* w, const void* 
 }
 
 int qes_update(const qes_tensor_desc* desc, void* w_inout, const void* scales_f16,
-               const uint64_t* seeds, const float* fitness, int32_t K, float* residual_inout,
+               const uint64_t* seeds, const float* fitness, int32_t K, void* residual_inout,
                const qes_hparams* hparams, uint64_t* stats, void* cuda_stream) {
     int rc = validate(desc, hparams);
     if (rc != QES_OK) return rc;

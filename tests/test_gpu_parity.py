@@ -345,3 +345,42 @@ def test_antithetic_pairs_update_replay_and_perturb(qo, qes, bits, rows, cols, N
     inplace = _dev(packed)
     qes.qes_perturb_pair(tg, inplace, inplace, wm, sc_d, seed, hg)       # the + output may alias the input
     assert np.array_equal(_host(inplace), _host(wp))
+
+
+def _half_spacing(x):
+    """Spacing of binary16 at |x| (2^-24 in the subnormal range)."""
+    a = np.maximum(np.abs(x), 2.0 ** -14)
+    return 2.0 ** (np.floor(np.log2(a)) - 10)
+
+
+def test_stored_residual_in_binary16(qo, qes):
+    """Algorithm 1 with the residual kept in FP16: three chained steps, each checked against the oracle started
+    from the library's own previous state; codes as usual, the stored residual must be a correct binary16
+    rounding of a value within 1e-5 of the oracle's."""
+    import torch
+    bits, rows, cols, N = 4, 29, 416, 8
+    to, tg, packed, _ = _case(qo, qes, bits, rows, cols, off=64)
+    n = rows * cols
+    kw = dict(sigma=0.5, lr=0.7, gamma=0.9, n_pop=N, residual_f16=1)
+    ho, hg = _hp(qo, qes, **kw)
+    w = _dev(packed)
+    e = torch.zeros(n, dtype=torch.float16, device="cuda")
+    for step in range(3):
+        w_before, e_before = _host(w).copy(), _host(e).copy()
+        seeds, fit = wl.draw_seeds(1, N, stream=200 + step), wl.draw_fitness(1, N, stream=200 + step)
+        qes.qes_update(tg, w, None, _dev(seeds), _dev(fit), 0, e, hg)
+        ref = qo.update(to, w_before, None, seeds, fit, 0, ho, residual_in=e_before)
+        _compare_update(qo, _host(w), bits, ref, f"fp16 residual, step {step}")
+        far = ref["band"] >= BAND
+        got = _host(e).astype(np.float64)
+        assert np.all(np.abs(got - ref["e_new"])[far] <= 0.5 * _half_spacing(ref["e_new"][far]) + TOL)
+        assert np.mean(_host(e).view(np.uint16)[far] == qo.to_half(ref["e_new"])[far]) > 0.995
+    assert np.any(_host(e) != 0)
+    # the history loop can write binary16 too
+    K = 3
+    seeds, fit = wl.draw_seeds(K, N, stream=210), wl.draw_fitness(K, N, stream=210)
+    out = torch.empty(n, dtype=torch.float16, device="cuda")
+    qes.qes_replay_residual(tg, _dev(packed), None, _dev(seeds), _dev(fit), K, hg, out)
+    rr = qo.replay_residual(to, packed, None, seeds, fit, K, ho)
+    far = rr["band"] >= BAND
+    assert np.all(np.abs(_host(out).astype(np.float64) - rr["e"])[far] <= 0.5 * _half_spacing(rr["e"][far]) + TOL)
