@@ -108,53 +108,69 @@ void bm24_cossin(uint32_t r1, float* c_out, float* s_out) {
 // 4-bit range of the perturbation tensor (App. A "4-bit stochastically rounded perturbation"):
 // [-8, 7], or the symmetric [-7, 7] (dmin = -7) when members come in antithetic pairs +-delta,
 // so that the mirrored member fits the same 4 bits.
-int stochastic_round_f32(float x, uint32_t rword, int dmin = -8) {
+int stochastic_round_exact(float x, double v, int dmin) {
     double xd = (double)x;
     double fl = std::floor(xd);
     double frac = xd - fl;                          // exact
-    double v = (double)(rword >> 8) / 16777216.0;   // exact, [0,1)
     int d = (int)fl + (v < frac ? 1 : 0);
     return std::min(7, std::max(dmin, d));
 }
 
-struct PairNoise { int delta[2]; double x[2]; bool near[2]; };
+// The default contract: v = (word >> 8) / 2^24.
+int stochastic_round_f32(float x, uint32_t rword, int dmin = -8) {
+    return stochastic_round_exact(x, (double)(rword >> 8) / 16777216.0, dmin);   // exact, [0,1)
+}
+
+struct Sample { int delta; double x; bool near; };
 
 const double kPi = 3.14159265358979323846;
 
-// Both discrete perturbations of pair p for one seed.  sig[] = sigma_eff of the
-// even and odd element.  tier 0 also flags samples whose decision lies within
-// tau of a floor boundary or of the Bernoulli threshold.
-PairNoise pair_noise(uint64_t seed, uint64_t p, const float sig[2], int tier, double tau, int dmin = -8) {
-    U4 r = philox4x32_10((uint32_t)p, (uint32_t)(p >> 32), 0u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32));
-    PairNoise out;
-    if (tier == 1) {
-        float R = bm24_radius(r.v[0]);
-        float cs, sn;
-        bm24_cossin(r.v[1], &cs, &sn);
-        float trig[2] = {cs, sn};
-        for (int h = 0; h < 2; ++h) {
-            float rho = sig[h] * R;
-            float x = rho * trig[h];
-            out.delta[h] = stochastic_round_f32(x, r.v[2 + h], dmin);
-            out.x[h] = (double)x;
-            out.near[h] = false;
-        }
+// The discrete perturbation of global element J for one seed.  Two ways of spending the 128 bits
+// of a Philox call (noise_mode):
+//   0  one call per PAIR of elements (counter = J >> 1): words 0,1 -> Box-Muller pair (cos for the
+//      even element, sin for the odd one), words 2,3 -> their 24-bit Bernoulli uniforms.
+//   1  one call per QUAD of elements (counter = J >> 2): words 0,1 -> Box-Muller pair for elements
+//      0,1 of the quad, words 2,3 -> pair for elements 2,3, each from the top 24 bits of its words
+//      as before; element h takes its Bernoulli uniform from the low byte b of word h (bits the
+//      Gaussian does not use): v = (b + 1/2) / 256, so that P(b = 1) is the fraction of x rounded
+//      to the nearest multiple of 1/256 (off Eq. 3's probability by at most 1/512).
+// tier 0 also flags samples whose decision lies within tau of a floor boundary or of the threshold.
+Sample sample_noise(uint64_t seed, uint64_t J, float sig, int tier, double tau, int dmin, int noise_mode) {
+    const uint64_t g = noise_mode ? (J >> 2) : (J >> 1);
+    U4 r = philox4x32_10((uint32_t)g, (uint32_t)(g >> 32), 0u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32));
+    const int odd = (int)(J & 1);
+    uint32_t w_radius, w_angle;
+    double v;
+    if (noise_mode == 0) {
+        w_radius = r.v[0]; w_angle = r.v[1];
+        v = (double)(r.v[2 + odd] >> 8) / 16777216.0;
     } else {
-        double u1 = (double)((r.v[0] >> 8) + 1u) / 16777216.0;
-        double u2 = (double)(r.v[1] >> 8) / 16777216.0;
+        const int h = (int)(J & 3);
+        w_radius = r.v[h & 2]; w_angle = r.v[(h & 2) + 1];
+        v = ((double)(r.v[h] & 0xffu) + 0.5) / 256.0;
+    }
+    Sample out;
+    if (tier == 1) {
+        float R = bm24_radius(w_radius);
+        float cs, sn;
+        bm24_cossin(w_angle, &cs, &sn);
+        float rho = sig * R;
+        float x = rho * (odd ? sn : cs);
+        out.delta = stochastic_round_exact(x, v, dmin);
+        out.x = (double)x;
+        out.near = false;
+    } else {
+        double u1 = (double)((w_radius >> 8) + 1u) / 16777216.0;
+        double u2 = (double)(w_angle >> 8) / 16777216.0;
         double R = std::sqrt(-2.0 * std::log(u1));
         double th = 2.0 * kPi * u2;
-        double trig[2] = {std::cos(th), std::sin(th)};
-        for (int h = 0; h < 2; ++h) {
-            double x = (double)sig[h] * R * trig[h];
-            double fl = std::floor(x);
-            double frac = x - fl;
-            double v = (double)(r.v[2 + h] >> 8) / 16777216.0;
-            int d = (int)fl + (v < frac ? 1 : 0);
-            out.delta[h] = std::min(7, std::max(dmin, d));
-            out.x[h] = x;
-            out.near[h] = (frac < tau) || (frac > 1.0 - tau) || (std::fabs(frac - v) < tau);
-        }
+        double x = (double)sig * R * (odd ? std::sin(th) : std::cos(th));
+        double fl = std::floor(x);
+        double frac = x - fl;
+        int d = (int)fl + (v < frac ? 1 : 0);
+        out.delta = std::min(7, std::max(dmin, d));
+        out.x = x;
+        out.near = (frac < tau) || (frac > 1.0 - tau) || (std::fabs(frac - v) < tau);
     }
     return out;
 }
@@ -213,7 +229,7 @@ struct Tensor { int32_t bits, qmin, qmax, group_size; int64_t rows, cols; uint64
 // generation, fitness holds n_pop entries per generation ordered F+_0, F-_0, F+_1, F-_1, ...
 // residual_f16 != 0: the stored residual of Algorithm 1 is kept in binary16 ("Residuals e_0 <- 0 (FP16)"):
 // read as binary16, all arithmetic as before; the caller rounds the returned e back to binary16.
-struct HParams { float sigma, lr, gamma; int32_t n_pop, sigma_unit, boundary_mode, antithetic, residual_f16; };
+struct HParams { float sigma, lr, gamma; int32_t n_pop, sigma_unit, boundary_mode, antithetic, residual_f16, noise_mode; };
 
 float sigma_eff(const Tensor& t, const HParams& hp, const uint16_t* scales, int64_t j) {
     if (hp.sigma_unit == 0) return hp.sigma;                    // sigma in grid steps
@@ -236,6 +252,7 @@ int check(const Tensor& t, const HParams& hp) {
     if (t.group_size < 0 || (t.group_size > 0 && t.cols % t.group_size)) return -3;
     if (!(hp.sigma > 0.f) || hp.n_pop <= 0 || !(hp.gamma >= 0.f && hp.gamma <= 1.f) || t.qmin >= t.qmax) return -5;
     if (hp.antithetic != 0 && hp.antithetic != 1) return -6;
+    if (hp.noise_mode != 0 && hp.noise_mode != 1) return -6;
     if (hp.antithetic && (hp.n_pop & 1)) return -5;
     return 0;
 }
@@ -259,12 +276,8 @@ struct ElemResult { int w_new; double e_new; double band; int gate_final; int ga
 ElemResult element_update(const Tensor& t, const HParams& hp, const uint16_t* scales, int w, int64_t j,
                           const uint64_t* seeds, const float* fitness, int gens, double e0,
                           bool replay_only, int tier) {
-    uint64_t J = t.elem_offset + (uint64_t)j;
-    uint64_t p = J >> 1;
-    int h = (int)(J & 1);
-    float sig[2];
-    sig[h] = sigma_eff(t, hp, scales, j);
-    sig[h ^ 1] = sig[h];
+    const uint64_t J = t.elem_offset + (uint64_t)j;
+    const float sig = sigma_eff(t, hp, scales, j);
     const int N = hp.n_pop;
     const double c = (double)hp.lr / ((double)N * (double)hp.sigma);
     const double gamma = (double)hp.gamma;
@@ -274,15 +287,15 @@ ElemResult element_update(const Tensor& t, const HParams& hp, const uint16_t* sc
         double S = 0.0;
         if (!hp.antithetic) {
             for (int i = 0; i < N; ++i) {
-                PairNoise pn = pair_noise(seeds[(int64_t)k * N + i], p, sig, tier, 0.0);
-                S += (double)fitness[(int64_t)k * N + i] * (double)pn.delta[h];   // Eq. 5 numerator
+                Sample sm = sample_noise(seeds[(int64_t)k * N + i], J, sig, tier, 0.0, -8, hp.noise_mode);
+                S += (double)fitness[(int64_t)k * N + i] * (double)sm.delta;      // Eq. 5 numerator
             }
         } else {
             // Eq. 5 over all N members, members 2j and 2j+1 carrying +delta_j and -delta_j
             for (int jp = 0; jp < N / 2; ++jp) {
-                PairNoise pn = pair_noise(seeds[(int64_t)k * (N / 2) + jp], p, sig, tier, 0.0, -7);
-                S += (double)fitness[(int64_t)k * N + 2 * jp] * (double)pn.delta[h];
-                S += (double)fitness[(int64_t)k * N + 2 * jp + 1] * (double)(-pn.delta[h]);
+                Sample sm = sample_noise(seeds[(int64_t)k * (N / 2) + jp], J, sig, tier, 0.0, -7, hp.noise_mode);
+                S += (double)fitness[(int64_t)k * N + 2 * jp] * (double)sm.delta;
+                S += (double)fitness[(int64_t)k * N + 2 * jp + 1] * (double)(-sm.delta);
             }
         }
         double u = c * S + gamma * e;                                          // Eq. 6
@@ -324,6 +337,9 @@ void qo_bm24(const uint32_t* r0, const uint32_t* r1, int64_t n, float* R, float*
 
 int qo_stochastic_round(float x, uint32_t rword) { return stochastic_round_f32(x, rword); }
 
+// Eq. 3 with the Bernoulli uniform of noise_mode 1: v = (byte + 1/2) / 256.
+int qo_stochastic_round_byte(float x, uint32_t byte) { return stochastic_round_exact(x, ((double)(byte & 0xffu) + 0.5) / 256.0, -8); }
+
 float qo_half_to_float(uint16_t h) { return half_to_float(h); }
 
 uint16_t qo_double_to_half(double v) { return double_to_half(v); }
@@ -335,14 +351,12 @@ void qo_doubles_to_halves(const double* v, int64_t n, uint16_t* out) {
 // delta (and optionally x = sigma_eff * eps, near-decision flags) of global
 // elements J[0..n) for one seed and one sigma_eff.
 void qo_delta(uint64_t seed, const uint64_t* J, int64_t n, float sigma_eff_v, int tier, double tau, int dmin,
-              int32_t* delta, double* x, uint8_t* near) {
-    float sig[2] = {sigma_eff_v, sigma_eff_v};
+              int noise_mode, int32_t* delta, double* x, uint8_t* near) {
     for (int64_t i = 0; i < n; ++i) {
-        PairNoise pn = pair_noise(seed, J[i] >> 1, sig, tier, tau, dmin);
-        int h = (int)(J[i] & 1);
-        delta[i] = pn.delta[h];
-        if (x) x[i] = pn.x[h];
-        if (near) near[i] = pn.near[h] ? 1 : 0;
+        Sample sm = sample_noise(seed, J[i], sigma_eff_v, tier, tau, dmin, noise_mode);
+        delta[i] = sm.delta;
+        if (x) x[i] = sm.x;
+        if (near) near[i] = sm.near ? 1 : 0;
     }
 }
 
@@ -367,12 +381,10 @@ int qo_perturb(const Tensor* t, const uint8_t* w, const uint16_t* scales, uint64
         for (int64_t i = lo; i < hi; ++i) {
             int64_t j = idx ? idx[i] : i;
             uint64_t J = t->elem_offset + (uint64_t)j;
-            int h = (int)(J & 1);
-            float sig[2];
-            sig[0] = sig[1] = sigma_eff(*t, *hp, scales, j);
-            PairNoise pn = pair_noise(seed, J >> 1, sig, tier, 0.0, hp->antithetic ? -7 : -8);
+            Sample sm = sample_noise(seed, J, sigma_eff(*t, *hp, scales, j), tier, 0.0, hp->antithetic ? -7 : -8,
+                                     hp->noise_mode);
             int code = load_code(w, t->bits, j);
-            w_out[i] = code + (int)applied_step(code, (long long)sign * pn.delta[h], t->qmin, t->qmax, hp->boundary_mode);
+            w_out[i] = code + (int)applied_step(code, (long long)sign * sm.delta, t->qmin, t->qmax, hp->boundary_mode);
         }
     });
     return 0;

@@ -40,7 +40,7 @@ class _Tensor(C.Structure):
 class _HParams(C.Structure):
     _fields_ = [("sigma", C.c_float), ("lr", C.c_float), ("gamma", C.c_float),
                 ("n_pop", C.c_int32), ("sigma_unit", C.c_int32), ("boundary_mode", C.c_int32),
-                ("antithetic", C.c_int32), ("residual_f16", C.c_int32)]
+                ("antithetic", C.c_int32), ("residual_f16", C.c_int32), ("noise_mode", C.c_int32)]
 
 
 @dataclass
@@ -73,10 +73,11 @@ class HParams:
     boundary_mode: int = 0   # 0 gate (Eq. 4), 1 clamp
     antithetic: int = 0      # 1: n_pop / 2 seeded pairs (+delta, -delta); fitness interleaved F+, F-
     residual_f16: int = 0    # 1: the stored residual is binary16
+    noise_mode: int = 0      # 0: one Philox call per two elements, 24-bit Bernoulli; 1: per four, 8-bit
 
     def c(self) -> _HParams:
         return _HParams(self.sigma, self.lr, self.gamma, self.n_pop, self.sigma_unit, self.boundary_mode,
-                        self.antithetic, self.residual_f16)
+                        self.antithetic, self.residual_f16, self.noise_mode)
 
 
 _lib = None
@@ -90,6 +91,8 @@ def lib() -> C.CDLL:
         _lib.qo_half_to_float.argtypes = [C.c_uint16]
         _lib.qo_stochastic_round.restype = C.c_int
         _lib.qo_stochastic_round.argtypes = [C.c_float, C.c_uint32]
+        _lib.qo_stochastic_round_byte.restype = C.c_int
+        _lib.qo_stochastic_round_byte.argtypes = [C.c_float, C.c_uint32]
         _lib.qo_double_to_half.restype = C.c_uint16
         _lib.qo_double_to_half.argtypes = [C.c_double]
         _lib.qo_applied_step.restype = C.c_longlong
@@ -126,6 +129,10 @@ def stochastic_round(x: float, rword: int) -> int:
     return lib().qo_stochastic_round(C.c_float(x), C.c_uint32(rword))
 
 
+def stochastic_round_byte(x: float, byte: int) -> int:
+    return lib().qo_stochastic_round_byte(C.c_float(x), C.c_uint32(byte))
+
+
 def half_to_float(h: int) -> float:
     return lib().qo_half_to_float(C.c_uint16(h))
 
@@ -142,14 +149,15 @@ def applied_step(w: int, step: int, qmin: int, qmax: int, mode: int) -> int:
     return lib().qo_applied_step(w, step, qmin, qmax, mode)
 
 
-def delta(seed: int, J, sigma_eff: float, tier: int = TIER_SPEC, tau: float = 0.0, dmin: int = -8):
+def delta(seed: int, J, sigma_eff: float, tier: int = TIER_SPEC, tau: float = 0.0, dmin: int = -8,
+          noise_mode: int = 0):
     """Discrete perturbation of global elements J for one seed: (delta int32, x float64, near uint8).
     dmin = -7 gives the symmetric 4-bit range used for antithetic pairs."""
     J = _arr(J, np.uint64)
     n = J.size
     d = np.empty(n, np.int32); x = np.empty(n, np.float64); near = np.empty(n, np.uint8)
     lib().qo_delta(C.c_uint64(seed), _p(J), C.c_int64(n), C.c_float(sigma_eff), C.c_int(tier),
-                   C.c_double(tau), C.c_int(dmin), _p(d), _p(x), _p(near))
+                   C.c_double(tau), C.c_int(dmin), C.c_int(noise_mode), _p(d), _p(x), _p(near))
     return d, x, near
 
 
