@@ -35,6 +35,8 @@ from paper_2602_03120_b200 import workloads as wl  # noqa: E402
 #                    polynomials 8, quadrant 4), sigma scaling 3                              = 42
 #   Eq. 3 + Eq. 5 per sample: floor, fraction, shift, compare, add, weighted fma = 7 (x2)    = 14
 OPS_PER_SAMPLE = (40 + 42 + 14) / 2.0
+# quad8: one Philox call (40) and two Box-Muller pairs (2 x 42) serve four samples (4 x 7)
+OPS_PER_SAMPLE_QUAD8 = (40 + 2 * 42 + 4 * 7) / 4.0
 OPS_PER_ELEM_GEN = 8.0      # u (2), round, w + step, two compares, select, residual
 OPS_PER_ELEM = 6.0          # unpack / repack
 SM_COUNT, LANES_PER_SM = 148, 128
@@ -44,8 +46,8 @@ SM_COUNT, LANES_PER_SM = 148, 128
 DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE = 0.80
 
 
-def alu_ops(numel: int, n_pop: int, generations: int) -> float:
-    return numel * (n_pop * generations * OPS_PER_SAMPLE + generations * OPS_PER_ELEM_GEN + OPS_PER_ELEM)
+def alu_ops(numel: int, n_pop: int, generations: int, per_sample: float = OPS_PER_SAMPLE) -> float:
+    return numel * (n_pop * generations * per_sample + generations * OPS_PER_ELEM_GEN + OPS_PER_ELEM)
 
 
 def measured_peaks():
@@ -94,7 +96,7 @@ class ClockSampler:
                 "power_w_max": max(pw) if pw else None, "samples": len(clk), "reasons": reasons}
 
 
-def oracle_rate(cfg: wl.Workload, target_seconds: float = 15.0, antithetic: bool = False):
+def oracle_rate(cfg: wl.Workload, target_seconds: float = 15.0, antithetic: bool = False, quad: bool = False):
     """Times the CPU oracle (as it stands) on a bounded sample of the workload: whole 32-element words
     drawn from the first tensor of the set, one full step on them (the perturbation of every member,
     then the stateless update) at the configuration's N and K.  Returns a dict."""
@@ -106,7 +108,8 @@ def oracle_rate(cfg: wl.Workload, target_seconds: float = 15.0, antithetic: bool
     n_seeds = cfg.n_pop // 2 if antithetic else cfg.n_pop
     seeds, fit = wl.draw_seeds(cfg.K + 1, n_seeds), wl.draw_fitness(cfg.K + 1, cfg.n_pop, cfg.reward_dist)
     to = qo.Tensor(bits=cfg.bits, rows=t.rows, cols=t.cols, group_size=cfg.group_size, elem_offset=t.elem_offset)
-    hp = qo.HParams(sigma=cfg.sigma, lr=cfg.lr, gamma=cfg.gamma, n_pop=cfg.n_pop, antithetic=int(antithetic))
+    hp = qo.HParams(sigma=cfg.sigma, lr=cfg.lr, gamma=cfg.gamma, n_pop=cfg.n_pop, antithetic=int(antithetic),
+                    noise_mode=int(quad))
     per_elem = n_seeds * (cfg.K + 1)
 
     def one_step(idx):
@@ -134,13 +137,13 @@ def run_reference(args, cfg):
     if rank != 0:
         return
     per_step = max(1.0, min(20.0, 150.0 / max(1, args.steps + args.warmup)))
-    rates = [oracle_rate(cfg, per_step, args.antithetic) for _ in range(args.warmup + args.steps)][args.warmup:]
+    rates = [oracle_rate(cfg, per_step, args.antithetic, args.noise_mode == "quad8") for _ in range(args.warmup + args.steps)][args.warmup:]
     tot_w = sum(r["elements"] for r in rates); tot_t = sum(r["seconds"] for r in rates)
     value = tot_w / tot_t
     line = {"impl": "reference", "metric": "weights_updated_per_s", "value": value, "unit": "weights/s",
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot_t / len(rates),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int4+f32" if cfg.bits == 4 else "int8+f32",
-            "data": "synthetic", "config": config_dict(cfg, args.gpus, args.antithetic),
+            "data": "synthetic", "config": config_dict(cfg, args.gpus, args.antithetic, args.noise_mode),
             "noise_samples_per_s": value * cfg.n_pop * (cfg.K + 1),
             "cpu_baseline": {"value": value, "unit": "weights/s", "cores": rates[0]["cores"], "kind": "oracle",
                              "sample": f"{rates[0]['elements']} elements (32-element words of tensor 0) per step, "
@@ -149,8 +152,8 @@ def run_reference(args, cfg):
     print(json.dumps(line))
 
 
-def config_dict(cfg, n_gpus, antithetic=False):
-    return {"population": "antithetic pairs" if antithetic else "independent members", "workload": cfg.name, "bits": cfg.bits, "weights_per_gpu": cfg.numel, "tensors_per_gpu": len(cfg.tensors),
+def config_dict(cfg, n_gpus, antithetic=False, noise_mode="pair24"):
+    return {"population": "antithetic pairs" if antithetic else "independent members", "noise_mode": noise_mode, "workload": cfg.name, "bits": cfg.bits, "weights_per_gpu": cfg.numel, "tensors_per_gpu": len(cfg.tensors),
             "n_pop": cfg.n_pop, "K": cfg.K, "sigma": cfg.sigma, "lr": cfg.lr, "gamma": cfg.gamma,
             "sigma_unit": "grid", "boundary": "gate", "perturb_members_per_step": cfg.n_pop,
             "launches": "one library call per run of consecutive tensors, at most 2^28 codes each",
@@ -169,6 +172,9 @@ def main():
     ap.add_argument("--antithetic", action="store_true",
                     help="the population is N/2 antithetic pairs (App. A): N/2 seeds per generation, both members of a "
                          "pair perturbed from one noise pass")
+    ap.add_argument("--noise-mode", default="pair24", choices=["pair24", "quad8"],
+                    help="pair24 (default): one Philox call per two elements, 24-bit Bernoulli uniforms; quad8: one call "
+                         "per four elements, 8-bit Bernoulli uniforms")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -196,7 +202,8 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    model = ModelPass(cfg, rank=rank, world=world, antithetic=args.antithetic)
+    quad = args.noise_mode == "quad8"
+    model = ModelPass(cfg, rank=rank, world=world, antithetic=args.antithetic, noise_mode=int(quad))
     n_seeds = cfg.n_pop // 2 if args.antithetic else cfg.n_pop
     host = torch.from_numpy(model.host_codes()).pin_memory()
     host_out = torch.empty_like(host).pin_memory()
@@ -283,30 +290,31 @@ def main():
 
     hbm_gbs, sm_mhz, peak_src = measured_peaks()
     G = cfg.K + 1
-    upd_ops_per_launch = alu_ops(model.numel, n_seeds, G) * args.steps / n_upd_launches
+    per_sample = OPS_PER_SAMPLE_QUAD8 if quad else OPS_PER_SAMPLE
+    upd_ops_per_launch = alu_ops(model.numel, n_seeds, G, per_sample) * args.steps / n_upd_launches
     upd_s_per_launch = update_ms * 1e-3 / n_upd_launches
     alu_peak = SM_COUNT * LANES_PER_SM * sm_mhz * 1e6
     achieved = upd_ops_per_launch / upd_s_per_launch
     bytes_per_launch = 2 * wl.packed_bytes(cfg.bits, model.numel) * args.steps / n_upd_launches
-    traffic = None if DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE is None else DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE * bytes_per_launch
+    traffic = None if (DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE is None or quad or args.antithetic) else DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE * bytes_per_launch
     roofline = {"bound": "alu", "kernel": f"pass_kernel<{cfg.bits}> (qes_update, stateless)",
                 "achieved": achieved / 1e9, "peak": alu_peak / 1e9, "unit": "Glane-op/s", "frac": achieved / alu_peak,
                 "peak_source": f"{SM_COUNT} SMs x 4 schedulers x 32 lanes x {sm_mhz:.0f} MHz (one instruction per scheduler "
                                f"per cycle; SM clock from the {peak_src} peaks file)",
-                "ops_per_sample": OPS_PER_SAMPLE, "avg_launch_ms": upd_s_per_launch * 1e3, "launches": n_upd_launches,
+                "ops_per_sample": per_sample, "avg_launch_ms": upd_s_per_launch * 1e3, "launches": n_upd_launches,
                 "traffic": traffic,
                 "hbm": {"achieved_gbs": bytes_per_launch / upd_s_per_launch / 1e9, "peak_gbs": hbm_gbs,
                         "frac": bytes_per_launch / upd_s_per_launch / 1e9 / hbm_gbs, "of": peak_src}}
     line = {"metric": "weights_updated_per_s", "value": value, "unit": "weights/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "int4+f32" if cfg.bits == 4 else "int8+f32",
-            "data": "synthetic", "config": config_dict(cfg, world, args.antithetic),
+            "data": "synthetic", "config": config_dict(cfg, world, args.antithetic, args.noise_mode),
             "noise_samples_per_s": world * model.numel * n_seeds * G / (update_ms * 1e-3 / args.steps),
             "update_ms_per_step": update_ms / args.steps, "perturb_ms_per_step": perturb_ms / args.steps,
             "perturb_weights_per_s": world * model.numel * cfg.n_pop / (perturb_ms * 1e-3 / args.steps),
             "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "e2e": e2e}
     if not args.no_cpu_baseline and world == 1:
-        r = oracle_rate(cfg, antithetic=args.antithetic)
+        r = oracle_rate(cfg, antithetic=args.antithetic, quad=quad)
         line["cpu_baseline"] = {"value": r["weights_per_s"], "unit": "weights/s", "cores": r["cores"], "kind": "oracle",
                                 "samples_per_s": r["samples_per_s"],
                                 "sample": f"{r['elements']} elements (32-element words of tensor 0), one full step (perturb x N, update), "

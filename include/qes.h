@@ -52,6 +52,14 @@ typedef enum {
 
 enum { QES_SIGMA_GRID = 0, QES_SIGMA_WEIGHT = 1 };   /* unit of hparams.sigma: grid steps | weight units (sigma_g = sigma / scale_g) */
 enum { QES_BOUNDARY_GATE = 0, QES_BOUNDARY_CLAMP = 1 }; /* Eq. 4 masking | saturation */
+/* How the 128 bits of one Philox4x32-10 call are spent (the paper leaves "RNG(seed)" open):
+ *   QES_NOISE_PAIR24  one call per two elements, counter = J >> 1: words 0,1 -> Box-Muller pair, words 2,3 ->
+ *                     24-bit Bernoulli uniforms of Eq. 3 (the default; P(b = 1) exact to 2^-24)
+ *   QES_NOISE_QUAD8   one call per four elements, counter = J >> 2: words 0,1 and 2,3 -> two Box-Muller pairs
+ *                     (top 24 bits of each word), element h's Bernoulli uniform (b + 1/2) / 256 from the low byte b
+ *                     of word h (P(b = 1) is the fraction of sigma*eps to the nearest 1/256); half the Philox work.
+ * The two modes draw different streams; each is reproduced bit for bit by the reference implementation. */
+enum { QES_NOISE_PAIR24 = 0, QES_NOISE_QUAD8 = 1 };
 
 typedef struct {
     int32_t bits;          /* 4 or 8 */
@@ -76,6 +84,7 @@ typedef struct {
     int32_t residual_f16;  /* format of residual_inout / residual_out: 0 = float, 1 = IEEE binary16 (Algorithm 1,
                               "Residuals e_0 <- 0 (FP16)"): read as binary16, arithmetic in fp32, rounded to
                               nearest even on the store */
+    int32_t noise_mode;    /* QES_NOISE_PAIR24 | QES_NOISE_QUAD8 */
 } qes_hparams;
 
 /*

@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libqes.so")
 
 SIGMA_GRID, SIGMA_WEIGHT = 0, 1
 BOUNDARY_GATE, BOUNDARY_CLAMP = 0, 1
+NOISE_PAIR24, NOISE_QUAD8 = 0, 1
 
 
 class QesError(RuntimeError):
@@ -31,7 +32,7 @@ class _TensorDesc(C.Structure):
 class _HParams(C.Structure):
     _fields_ = [("sigma", C.c_float), ("lr", C.c_float), ("gamma", C.c_float),
                 ("n_pop", C.c_int32), ("sigma_unit", C.c_int32), ("boundary_mode", C.c_int32),
-                ("antithetic", C.c_int32), ("residual_f16", C.c_int32)]
+                ("antithetic", C.c_int32), ("residual_f16", C.c_int32), ("noise_mode", C.c_int32)]
 
 
 @dataclass
@@ -68,10 +69,11 @@ class HParams:
     boundary_mode: int = BOUNDARY_GATE
     antithetic: int = 0
     residual_f16: int = 0
+    noise_mode: int = NOISE_PAIR24
 
     def c(self) -> _HParams:
         return _HParams(self.sigma, self.lr, self.gamma, self.n_pop, self.sigma_unit, self.boundary_mode,
-                        self.antithetic, self.residual_f16)
+                        self.antithetic, self.residual_f16, self.noise_mode)
 
     @property
     def residual_dtype(self):

@@ -141,32 +141,33 @@ __device__ __forceinline__ int applied_code(int w, int step, int qmin, int qmax,
 // Algorithm 1, member loop: W' = Gate(W + delta_i), and with PAIR also the antithetic member
 // Gate(W - delta_i) from the same noise.  The member's round keys are computed on the host and
 // arrive as kernel parameters, i.e. as constant-bank operands.
-template <int BITS, bool CLAMP_DELTA, bool PAIR>
+template <int BITS, bool CLAMP_DELTA, bool PAIR, bool QUAD>
 __global__ void __launch_bounds__(kThreads) perturb_kernel(PassParams p, RoundKeys rk) {
+    constexpr int kPerCall = QUAD ? 4 : 2;                 // elements served by one Philox call
+    constexpr int kCalls = kCodesPerThread / kPerCall;
     int64_t chunk = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (chunk >= p.n_chunks) return;
     Chunk<BITS, kPairs> w;
     w.load(p.w_in, chunk);
     float nsig24 = chunk_neg_sigma24(p, chunk);
-    uint64_t pair0 = (p.elem_offset >> 1) + (uint64_t)chunk * kPairs;
-    uint32_t x0 = (uint32_t)pair0, y = (uint32_t)(pair0 >> 32);
+    uint64_t call0 = (p.elem_offset >> (QUAD ? 2 : 1)) + (uint64_t)chunk * kCalls;
+    uint32_t x0 = (uint32_t)call0, y = (uint32_t)(call0 >> 32);
     SeedConst sc = make_seed_const(y, rk);
     Chunk<BITS, kPairs> out, out_minus;
     out.clear();
     out_minus.clear();
 #pragma unroll
-    for (int i = 0; i < kPairs; ++i) {
+    for (int i = 0; i < kCalls; ++i) {
         uint32_t r0, r1, r2, r3;
         philox_tail(make_pair_const(x0 + i), sc, rk, r0, r1, r2, r3);
-        int z0, z1;
-        pair_rounding_sums<CLAMP_DELTA>(r0, r1, r2, r3, nsig24, z0, z1);
-        int nd0 = neg_delta<CLAMP_DELTA>(z0, p.nd_max), nd1 = neg_delta<CLAMP_DELTA>(z1, p.nd_max);
-        int w0 = w.get(2 * i), w1 = w.get(2 * i + 1);
-        out.put(2 * i, applied_code(w0, -nd0, p.qmin_i, p.qmax_i, p.boundary_mode));
-        out.put(2 * i + 1, applied_code(w1, -nd1, p.qmin_i, p.qmax_i, p.boundary_mode));
-        if (PAIR) {
-            out_minus.put(2 * i, applied_code(w0, nd0, p.qmin_i, p.qmax_i, p.boundary_mode));
-            out_minus.put(2 * i + 1, applied_code(w1, nd1, p.qmin_i, p.qmax_i, p.boundary_mode));
+        int z[kPerCall];
+        call_rounding_sums<CLAMP_DELTA, QUAD>(r0, r1, r2, r3, nsig24, z);
+#pragma unroll
+        for (int j = 0; j < kPerCall; ++j) {
+            const int t = kPerCall * i + j;
+            const int nd = neg_delta<CLAMP_DELTA>(z[j], p.nd_max), wc = w.get(t);
+            out.put(t, applied_code(wc, -nd, p.qmin_i, p.qmax_i, p.boundary_mode));
+            if (PAIR) out_minus.put(t, applied_code(wc, nd, p.qmin_i, p.qmax_i, p.boundary_mode));
         }
     }
     out.store(p.w_out, chunk);
@@ -210,10 +211,12 @@ __device__ __forceinline__ RoundKeys load_round_keys(const uint32_t* entry, floa
 
 // Algorithm 2 (stateless), Algorithm 1's update lines (stored residual) or the history loop
 // alone (replay only), selected by p.mode.  Shared memory: 2 * n_pop * 96 B.
-template <int BITS, bool CLAMP_DELTA, bool STATS>
+template <int BITS, bool CLAMP_DELTA, bool STATS, bool QUAD>
 __global__ void __launch_bounds__(kThreads, QES_MIN_BLOCKS) pass_kernel(PassParams p) {
     extern __shared__ __align__(16) uint32_t smem[];
     constexpr int T = kCodesPerThread;
+    constexpr int kPerCall = QUAD ? 4 : 2;                 // elements served by one Philox call
+    constexpr int kCalls = T / kPerCall;
     const int64_t chunk = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const bool active = chunk < p.n_chunks;
 
@@ -223,17 +226,17 @@ __global__ void __launch_bounds__(kThreads, QES_MIN_BLOCKS) pass_kernel(PassPara
 #pragma unroll
     for (int t = 0; t < T; ++t) e[t] = 0.0f;
     float nsig24 = 0.0f;
-    PairConst pc[kPairs];
+    PairConst pc[kCalls];
     uint32_t y = 0u;
     if (active) {
         w.load(p.w_in, chunk);
         if (p.mode == kStoredResidual) load_residual<T>(p.residual, p.residual_f16 != 0, chunk, e);
         nsig24 = chunk_neg_sigma24(p, chunk);
-        // a thread's pairs share the counter high word: pair0 is a multiple of kPairs
-        const uint64_t pair0 = (p.elem_offset >> 1) + (uint64_t)chunk * kPairs;
-        y = (uint32_t)(pair0 >> 32);
+        // a thread's calls share the counter high word: call0 is a multiple of kCalls
+        const uint64_t call0 = (p.elem_offset >> (QUAD ? 2 : 1)) + (uint64_t)chunk * kCalls;
+        y = (uint32_t)(call0 >> 32);
 #pragma unroll
-        for (int i = 0; i < kPairs; ++i) pc[i] = make_pair_const((uint32_t)pair0 + i);
+        for (int i = 0; i < kCalls; ++i) pc[i] = make_pair_const((uint32_t)call0 + i);
     }
 
     const int last = p.generations - 1;
@@ -243,11 +246,11 @@ __global__ void __launch_bounds__(kThreads, QES_MIN_BLOCKS) pass_kernel(PassPara
     Chunk<BITS, kPairs> out;
     out.clear();
 
-    // counter high word of the CTA's first pair; a CTA spans 256 * kPairs pairs, so at most one
-    // CTA in 2^32 / (256 * kPairs) sees a second value, and then its threads rebuild SeedConst
-    const uint64_t cta_pair0 = (p.elem_offset >> 1) + (uint64_t)blockIdx.x * (kThreads * kPairs);
-    const uint32_t y_cta = (uint32_t)(cta_pair0 >> 32);
-    const bool y_uniform = (uint32_t)((cta_pair0 + (uint64_t)(kThreads * kPairs - 1)) >> 32) == y_cta;
+    // counter high word of the CTA's first call; a CTA spans 256 * kCalls counters, so at most one
+    // CTA in 2^32 / (256 * kCalls) sees a second value, and then its threads rebuild SeedConst
+    const uint64_t cta_call0 = (p.elem_offset >> (QUAD ? 2 : 1)) + (uint64_t)blockIdx.x * (kThreads * kCalls);
+    const uint32_t y_cta = (uint32_t)(cta_call0 >> 32);
+    const bool y_uniform = (uint32_t)((cta_call0 + (uint64_t)(kThreads * kCalls - 1)) >> 32) == y_cta;
 
     if (p.generations > 0) stage_generation(smem, p.seeds, p.fitness, p.n_seeds, p.antithetic != 0, y_cta);
     for (int k = 0; k < p.generations; ++k) {
@@ -267,13 +270,14 @@ __global__ void __launch_bounds__(kThreads, QES_MIN_BLOCKS) pass_kernel(PassPara
             const RoundKeys rk = load_round_keys(table + i * kSeedStride, Fm, sc);
             if (!y_uniform) sc = make_seed_const(y, rk);
 #pragma unroll
-            for (int pr = 0; pr < kPairs; ++pr) {
+            for (int c = 0; c < kCalls; ++c) {
                 uint32_t r0, r1, r2, r3;
-                philox_tail(pc[pr], sc, rk, r0, r1, r2, r3);
-                int z0, z1;
-                pair_rounding_sums<CLAMP_DELTA>(r0, r1, r2, r3, nsig24, z0, z1);
-                S[2 * pr] = fmaf(Fm, neg_delta_scaled<CLAMP_DELTA>(z0, p.nd_max), S[2 * pr]);            // Eq. 5 numerator
-                S[2 * pr + 1] = fmaf(Fm, neg_delta_scaled<CLAMP_DELTA>(z1, p.nd_max), S[2 * pr + 1]);
+                philox_tail(pc[c], sc, rk, r0, r1, r2, r3);
+                int z[kPerCall];
+                call_rounding_sums<CLAMP_DELTA, QUAD>(r0, r1, r2, r3, nsig24, z);
+#pragma unroll
+                for (int j = 0; j < kPerCall; ++j)          // Eq. 5 numerator
+                    S[kPerCall * c + j] = fmaf(Fm, neg_delta_scaled<CLAMP_DELTA>(z[j], p.nd_max), S[kPerCall * c + j]);
             }
         }
         const bool is_update = (k == last) && (p.mode != kReplayOnly);
@@ -348,6 +352,7 @@ int validate(const qes_tensor_desc* d, const qes_hparams* h) {
     if (!(h->sigma > 0.0f) || !(h->sigma < 1e30f) || h->n_pop <= 0) return QES_ERR_BAD_HPARAM;
     if (h->antithetic != 0 && h->antithetic != 1) return QES_ERR_BAD_MODE;
     if (h->residual_f16 != 0 && h->residual_f16 != 1) return QES_ERR_BAD_MODE;
+    if (h->noise_mode != QES_NOISE_PAIR24 && h->noise_mode != QES_NOISE_QUAD8) return QES_ERR_BAD_MODE;
     if (h->antithetic && (h->n_pop & 1)) return QES_ERR_BAD_HPARAM;
     if (!(h->gamma >= 0.0f && h->gamma <= 1.0f) || !(h->lr == h->lr)) return QES_ERR_BAD_HPARAM;
     if (h->sigma_unit != QES_SIGMA_GRID && h->sigma_unit != QES_SIGMA_WEIGHT) return QES_ERR_BAD_MODE;
@@ -386,27 +391,28 @@ bool delta_clamp_needed(const qes_hparams* h) {
 
 size_t stage_bytes(int n_seeds) { return (size_t)2 * (size_t)n_seeds * kSeedStride * sizeof(uint32_t); }
 
-template <int BITS, bool CLAMP, bool STATS>
+template <int BITS, bool CLAMP, bool STATS, bool QUAD>
 int launch_pass(const PassParams& p, cudaStream_t stream) {
     const size_t smem = stage_bytes(p.n_seeds);
     if (smem > 48 * 1024) {
-        cudaError_t a = cudaFuncSetAttribute(pass_kernel<BITS, CLAMP, STATS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t a = cudaFuncSetAttribute(pass_kernel<BITS, CLAMP, STATS, QUAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (a != cudaSuccess) { cudaGetLastError(); return QES_ERR_CUDA; }
     }
     unsigned blocks = (unsigned)((p.n_chunks + kThreads - 1) / kThreads);
-    pass_kernel<BITS, CLAMP, STATS><<<blocks, kThreads, smem, stream>>>(p);
+    pass_kernel<BITS, CLAMP, STATS, QUAD><<<blocks, kThreads, smem, stream>>>(p);
     return cudaGetLastError() == cudaSuccess ? QES_OK : QES_ERR_CUDA;
 }
 
-template <int BITS>
+template <int BITS, bool QUAD>
 int dispatch_flags(bool clamp, bool stats, const PassParams& p, cudaStream_t stream) {
-    if (clamp) return stats ? launch_pass<BITS, true, true>(p, stream) : launch_pass<BITS, true, false>(p, stream);
-    return stats ? launch_pass<BITS, false, true>(p, stream) : launch_pass<BITS, false, false>(p, stream);
+    if (clamp) return stats ? launch_pass<BITS, true, true, QUAD>(p, stream) : launch_pass<BITS, true, false, QUAD>(p, stream);
+    return stats ? launch_pass<BITS, false, true, QUAD>(p, stream) : launch_pass<BITS, false, false, QUAD>(p, stream);
 }
 
-int dispatch_pass(int bits, bool clamp, const PassParams& p, cudaStream_t stream) {
+int dispatch_pass(int bits, bool clamp, bool quad, const PassParams& p, cudaStream_t stream) {
     const bool stats = p.stats != nullptr;
-    return bits == 4 ? dispatch_flags<4>(clamp, stats, p, stream) : dispatch_flags<8>(clamp, stats, p, stream);
+    if (quad) return bits == 4 ? dispatch_flags<4, true>(clamp, stats, p, stream) : dispatch_flags<8, true>(clamp, stats, p, stream);
+    return bits == 4 ? dispatch_flags<4, false>(clamp, stats, p, stream) : dispatch_flags<8, false>(clamp, stats, p, stream);
 }
 
 int check_table(const uint64_t* seeds, const float* fitness, int64_t generations, const qes_hparams* h) {
@@ -419,14 +425,14 @@ int check_table(const uint64_t* seeds, const float* fitness, int64_t generations
     return QES_OK;
 }
 
-template <int BITS>
+template <int BITS, bool QUAD>
 void launch_perturb_bits(bool clamp, bool pair, const PassParams& p, const RoundKeys& rk, unsigned blocks, cudaStream_t stream) {
     if (clamp) {
-        if (pair) perturb_kernel<BITS, true, true><<<blocks, kThreads, 0, stream>>>(p, rk);
-        else perturb_kernel<BITS, true, false><<<blocks, kThreads, 0, stream>>>(p, rk);
+        if (pair) perturb_kernel<BITS, true, true, QUAD><<<blocks, kThreads, 0, stream>>>(p, rk);
+        else perturb_kernel<BITS, true, false, QUAD><<<blocks, kThreads, 0, stream>>>(p, rk);
     } else {
-        if (pair) perturb_kernel<BITS, false, true><<<blocks, kThreads, 0, stream>>>(p, rk);
-        else perturb_kernel<BITS, false, false><<<blocks, kThreads, 0, stream>>>(p, rk);
+        if (pair) perturb_kernel<BITS, false, true, QUAD><<<blocks, kThreads, 0, stream>>>(p, rk);
+        else perturb_kernel<BITS, false, false, QUAD><<<blocks, kThreads, 0, stream>>>(p, rk);
     }
 }
 
@@ -451,8 +457,14 @@ int launch_perturb(const qes_tensor_desc* desc, const void* w_in, void* w_out, v
         rk.b[r] = (uint32_t)(seed >> 32) + kPhiloxW1 * (uint32_t)r;
     }
     const bool clamp = delta_clamp_needed(hparams);
-    if (desc->bits == 4) launch_perturb_bits<4>(clamp, w_minus != nullptr, p, rk, blocks, stream);
-    else launch_perturb_bits<8>(clamp, w_minus != nullptr, p, rk, blocks, stream);
+    const bool pair = w_minus != nullptr;
+    if (hparams->noise_mode == QES_NOISE_QUAD8) {
+        if (desc->bits == 4) launch_perturb_bits<4, true>(clamp, pair, p, rk, blocks, stream);
+        else launch_perturb_bits<8, true>(clamp, pair, p, rk, blocks, stream);
+    } else {
+        if (desc->bits == 4) launch_perturb_bits<4, false>(clamp, pair, p, rk, blocks, stream);
+        else launch_perturb_bits<8, false>(clamp, pair, p, rk, blocks, stream);
+    }
     return cudaGetLastError() == cudaSuccess ? QES_OK : QES_ERR_CUDA;
 }
 
@@ -493,7 +505,8 @@ int qes_replay_residual(const qes_tensor_desc* desc, const void* w, const void* 
     p.residual = residual_out;
     p.generations = K;
     p.mode = kReplayOnly;
-    return dispatch_pass(desc->bits, delta_clamp_needed(hparams), p, reinterpret_cast<cudaStream_t>(cuda_stream));
+    return dispatch_pass(desc->bits, delta_clamp_needed(hparams), hparams->noise_mode == QES_NOISE_QUAD8, p,
+                         reinterpret_cast<cudaStream_t>(cuda_stream));
 }
 
 int qes_update(const qes_tensor_desc* desc, void* w_inout, const void* scales_f16,
@@ -518,7 +531,8 @@ int qes_update(const qes_tensor_desc* desc, void* w_inout, const void* scales_f1
     p.stats = reinterpret_cast<unsigned long long*>(stats);
     p.generations = K + 1;
     p.mode = residual_inout != nullptr ? kStoredResidual : kStateless;
-    return dispatch_pass(desc->bits, delta_clamp_needed(hparams), p, reinterpret_cast<cudaStream_t>(cuda_stream));
+    return dispatch_pass(desc->bits, delta_clamp_needed(hparams), hparams->noise_mode == QES_NOISE_QUAD8, p,
+                         reinterpret_cast<cudaStream_t>(cuda_stream));
 }
 
 int qes_gaussian_factors(const uint32_t* r0, const uint32_t* r1, int64_t n, float* radius, float* cosine,

@@ -47,7 +47,7 @@ def launch_segments(tensors, max_elems: int = MAX_SEGMENT_ELEMS):
 class ModelPass:
     def __init__(self, workload: wl.Workload, device="cuda", rank: int = 0, world: int = 1,
                  sigma_unit: int = qes.SIGMA_GRID, with_scales: bool = False, tensors=None,
-                 antithetic: bool = False):
+                 antithetic: bool = False, noise_mode: int = qes.NOISE_PAIR24):
         self.wl = workload
         self.device = torch.device(device)
         self.tensors = tuple(tensors) if tensors is not None else shard_tensors(workload, rank, world)
@@ -56,7 +56,7 @@ class ModelPass:
         self.bytes = wl.packed_bytes(workload.bits, self.numel)
         self.w = torch.empty(self.bytes, dtype=torch.uint8, device=self.device)
         self.hp = qes.HParams(sigma=workload.sigma, lr=workload.lr, gamma=workload.gamma, n_pop=workload.n_pop,
-                              sigma_unit=sigma_unit, antithetic=int(antithetic))
+                              sigma_unit=sigma_unit, antithetic=int(antithetic), noise_mode=noise_mode)
         self.descs = [qes.TensorDesc(bits=workload.bits, rows=t.rows, cols=t.cols, group_size=workload.group_size,
                                      elem_offset=t.elem_offset) for t in self.tensors]
         # grid-unit sigma: fused launches over runs of tensors; weight-unit sigma: one launch per tensor

@@ -28,7 +28,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_struct_layouts_match_header():
     from paper_2602_03120_b200 import binding
-    assert C.sizeof(binding._TensorDesc) == 40 and C.sizeof(binding._HParams) == 32
+    assert C.sizeof(binding._TensorDesc) == 40 and C.sizeof(binding._HParams) == 36
     assert binding._TensorDesc.rows.offset == 16 and binding._TensorDesc.elem_offset.offset == 32
 
 
@@ -61,6 +61,8 @@ def test_invalid_arguments_are_rejected_without_launching(lib):
     # antithetic pairs: flag must be 0 or 1, the population even, the pair call needs the flag and two outputs
     ha = lambda **kw: binding.HParams(**{**dict(sigma=0.5, lr=1.0, gamma=0.9, n_pop=4, antithetic=1), **kw}).c()
     h2, h3, h1 = ha(antithetic=2), ha(n_pop=3), ha()
+    h5 = ha(antithetic=0, noise_mode=2)
+    assert lib.qes_update(C.byref(d), 0x1000, None, 0x2000, 0x3000, 1, None, C.byref(h5), None, None) == -6
     h4 = ha(antithetic=0, residual_f16=3)
     assert lib.qes_update(C.byref(d), 0x1000, None, 0x2000, 0x3000, 0, 0x4000, C.byref(h4), None, None) == -6
     assert lib.qes_update(C.byref(d), 0x1000, None, 0x2000, 0x3000, 1, None, C.byref(h2), None, None) == -6

@@ -384,3 +384,71 @@ def test_stored_residual_in_binary16(qo, qes):
     rr = qo.replay_residual(to, packed, None, seeds, fit, K, ho)
     far = rr["band"] >= BAND
     assert np.all(np.abs(_host(out).astype(np.float64) - rr["e"])[far] <= 0.5 * _half_spacing(rr["e"][far]) + TOL)
+
+
+@pytest.mark.parametrize("bits,rows,cols,off,N,K,sigma,mode,anti,unit", [
+    (4, 53, 608, 32 * 9, 8, 4, 0.5, 0, 0, 0), (8, 19, 352, (1 << 34) - 1024, 5, 2, 0.5, 1, 0, 0),
+    (4, 7, 1024, (1 << 34) - 2048, 6, 3, 2.0, 0, 1, 0), (4, 13, 384, (1 << 41) + 96, 4, 1, 0.012, 0, 0, 1),
+    (8, 1, 32, 0, 1, 0, 0.5, 0, 0, 0)])
+def test_quad_noise_mode(qo, qes, bits, rows, cols, off, N, K, sigma, mode, anti, unit):
+    """noise_mode = QUAD8 (one Philox call per four elements, 8-bit Bernoulli uniforms): perturbation, stateless
+    update, history loop and stored residual against the oracle in the same mode, including tensors that
+    straddle element 2^34, where the counter high word of this mode changes."""
+    import torch
+    group = 128 if (bits == 4 and unit) else 0
+    to, tg, packed, scales = _case(qo, qes, bits, rows, cols, group=group, off=off)
+    lr = 2.0 * sigma if unit else 1.0
+    kw = dict(sigma=sigma, lr=lr, gamma=0.9, n_pop=N, boundary_mode=mode, sigma_unit=unit, antithetic=anti, noise_mode=1)
+    ho, hg = _hp(qo, qes, **kw)
+    sc_d, sc_o = (_dev(scales), scales) if unit else (None, None)
+    n_seeds = N // 2 if anti else N
+    seeds, fit = wl.draw_seeds(K + 1, n_seeds, stream=300 + rows), wl.draw_fitness(K + 1, N, stream=300 + rows)
+    seed = int(seeds[-1, 0])
+    wp = _dev(np.zeros_like(packed))
+    qes.qes_perturb(tg, _dev(packed), wp, sc_d, seed, hg)
+    assert np.array_equal(_host(wp), qo.pack(bits, qo.perturb(to, packed, sc_o, seed, ho)))
+    if anti:
+        wm = _dev(np.zeros_like(packed))
+        qes.qes_perturb_pair(tg, _dev(packed), wp, wm, sc_d, seed, hg)
+        assert np.array_equal(_host(wm), qo.pack(bits, qo.perturb(to, packed, sc_o, seed, ho, sign=-1)))
+    w = _dev(packed)
+    stats = torch.zeros(4, dtype=torch.int64, device="cuda")
+    qes.qes_update(tg, w, sc_d, _dev(seeds), _dev(fit), K, None, hg, stats=stats)
+    ref = qo.update(to, packed, sc_o, seeds, fit, K, ho)
+    n_near = _compare_update(qo, _host(w), bits, ref, "quad noise update")
+    assert abs(int(_host(stats)[0]) - int((ref["w_new"] != qo.unpack(bits, packed, rows * cols)).sum())) <= n_near
+    plain = qo.update(to, packed, sc_o, seeds, fit, K, qo.HParams(**{**kw, "noise_mode": 0}))
+    if rows * cols > 1000:
+        assert not np.array_equal(plain["w_new"], ref["w_new"])          # the two modes are different streams
+    res = torch.empty(rows * cols, dtype=torch.float32, device="cuda")
+    qes.qes_replay_residual(tg, _dev(packed), sc_d, _dev(seeds[:K]), _dev(fit[:K]), K, hg, res)
+    rr = qo.replay_residual(to, packed, sc_o, seeds[:K], fit[:K], K, ho)
+    far = rr["band"] >= BAND
+    assert np.abs(_host(res).astype(np.float64) - rr["e"])[far].max(initial=0.0) <= TOL
+    e_in = np.random.default_rng(rows).uniform(-0.5, 0.5, rows * cols).astype(np.float32)
+    w2, e2 = _dev(packed), _dev(e_in)
+    qes.qes_update(tg, w2, sc_d, _dev(seeds[-1:]), _dev(fit[-1:]), 0, e2, hg)
+    ref2 = qo.update(to, packed, sc_o, seeds[-1:], fit[-1:], 0, ho, residual_in=e_in)
+    _compare_update(qo, _host(w2), bits, ref2, "quad noise stored residual")
+    far2 = ref2["band"] >= BAND
+    assert np.abs(_host(e2).astype(np.float64) - ref2["e_new"])[far2].max(initial=0.0) <= TOL
+
+
+def test_quad_noise_full_size_tensor_sampled(qo, qes):
+    """A full-size tensor of the 7B-shaped set in QUAD8 mode at the benchmark's N and K, oracle on sampled words."""
+    cfg = wl.WORKLOADS["decoder7b_int4"]
+    ti = 6
+    t = cfg.tensors[ti]
+    kw = dict(sigma=cfg.sigma, lr=cfg.lr, gamma=cfg.gamma, n_pop=cfg.n_pop, noise_mode=1)
+    ho, hg = _hp(qo, qes, **kw)
+    seeds, fit = wl.draw_seeds(cfg.K + 1, cfg.n_pop), wl.draw_fitness(cfg.K + 1, cfg.n_pop, cfg.reward_dist)
+    packed = wl.draw_codes(cfg, ti)
+    to = qo.Tensor(bits=4, rows=t.rows, cols=t.cols, group_size=cfg.group_size, elem_offset=t.elem_offset)
+    tg = qes.TensorDesc(bits=4, rows=t.rows, cols=t.cols, group_size=cfg.group_size, elem_offset=t.elem_offset)
+    w = _dev(packed)
+    qes.qes_update(tg, w, None, _dev(seeds), _dev(fit), cfg.K, None, hg)
+    idx = wl.sample_elements(t.numel, 2048, stream=77)
+    ref = qo.update(to, packed, None, seeds, fit, cfg.K, ho, idx=idx)
+    got = qo.unpack(4, _host(w), t.numel)[idx]
+    near = ref["band"] < BAND
+    assert not np.any((got != ref["w_new"]) & ~near)
