@@ -452,3 +452,70 @@ def test_quad_noise_full_size_tensor_sampled(qo, qes):
     got = qo.unpack(4, _host(w), t.numel)[idx]
     near = ref["band"] < BAND
     assert not np.any((got != ref["w_new"]) & ~near)
+
+
+@pytest.mark.parametrize("N,anti", [(600, 0), (1066, 0), (2132, 1)])
+def test_large_populations_stage_more_than_48_kib(qo, qes, N, anti):
+    """Populations whose staged round keys need the opt-in shared-memory size (96 B per seed, two
+    generations): 600 seeds = 112.5 KiB, and the documented maximum of 1066 seeds (or pairs)."""
+    bits, rows, cols, K = 4, 3, 128, 1
+    to, tg, packed, _ = _case(qo, qes, bits, rows, cols, off=96)
+    ho, hg = _hp(qo, qes, sigma=0.5, lr=1.0, gamma=0.9, n_pop=N, antithetic=anti)
+    n_seeds = N // 2 if anti else N
+    seeds, fit = wl.draw_seeds(K + 1, n_seeds, stream=N), wl.draw_fitness(K + 1, N, stream=N)
+    w = _dev(packed)
+    qes.qes_update(tg, w, None, _dev(seeds), _dev(fit), K, None, hg)
+    ref = qo.update(to, packed, None, seeds, fit, K, ho)
+    _compare_update(qo, _host(w), bits, ref, f"N = {N}")
+    too_many = qes.HParams(sigma=0.5, lr=1.0, gamma=0.9, n_pop=1067 * (2 if anti else 1), antithetic=anti)
+    with pytest.raises(qes.QesError):
+        qes.qes_update(tg, w, None, _dev(np.zeros(4 * 1067, np.uint64)), _dev(np.zeros(4 * 1067, np.float32)), 1, None, too_many)
+
+
+def test_model_pass_with_weight_unit_sigma_launches_per_tensor(qo, qes):
+    """ModelPass with sigma in weight units: one call per tensor, each with its own group scales."""
+    from paper_2602_03120_b200.model_pass import ModelPass
+    cfg = wl.WORKLOADS["decoder1p5b_int4"]
+    picks = (1, 2)                                         # k_proj, v_proj of layer 0: 256 x 1536 each
+    tensors = [cfg.tensors[i] for i in picks]
+    model = ModelPass(cfg, tensors=tensors, sigma_unit=qes.SIGMA_WEIGHT)
+    model.hp.sigma, model.hp.lr = 0.012, 0.024
+    model.scales = [_dev(wl.draw_scales(cfg, i)) for i in picks]
+    host = np.concatenate([wl.draw_codes(cfg, i) for i in picks])
+    model.load(host)
+    seeds, fit = wl.draw_seeds(cfg.K + 1, cfg.n_pop), wl.draw_fitness(cfg.K + 1, cfg.n_pop)
+    assert model.update(_dev(seeds), _dev(fit), cfg.K) == 2
+    got = _host(model.w)
+    ho = qo.HParams(sigma=0.012, lr=0.024, gamma=cfg.gamma, n_pop=cfg.n_pop, sigma_unit=1)
+    lo = 0
+    for i in picks:
+        t = cfg.tensors[i]
+        to = qo.Tensor(bits=4, rows=t.rows, cols=t.cols, group_size=cfg.group_size, elem_offset=t.elem_offset)
+        idx = wl.sample_elements(t.numel, 4096, stream=i)
+        ref = qo.update(to, wl.draw_codes(cfg, i), wl.draw_scales(cfg, i), seeds, fit, cfg.K, ho, idx=idx)
+        g = qo.unpack(4, got[lo:lo + t.numel // 2], t.numel)[idx]
+        assert not np.any((g != ref["w_new"]) & (ref["band"] >= BAND))
+        lo += t.numel // 2
+
+
+def test_resume_from_weights_and_history_through_the_library(qo, qes):
+    """Checkpoint / resume: the optimizer state is the packed weights plus the seed/reward window."""
+    from paper_2602_03120_b200.history import SeedHistory
+    N, K, T = 6, 3, 6
+    tg = qes.TensorDesc(bits=4, rows=16, cols=256)
+    hg = qes.HParams(sigma=0.5, lr=1.0, gamma=0.9, n_pop=N)
+    w0 = np.random.default_rng(9).integers(0, 256, 2048, dtype=np.uint8)
+    gens = [(wl.draw_seeds(1, N, stream=600 + s)[0], wl.draw_fitness(1, N, stream=600 + s)[0]) for s in range(T)]
+
+    def run(w_host, hist, steps):
+        w = _dev(w_host)
+        for s, f in steps:
+            seeds, fit, k = hist.tables(s, f)
+            qes.qes_update(tg, w, None, _dev(seeds), _dev(fit), k, None, hg)
+            hist.push(s, f)
+        return _host(w), hist
+
+    w_full, _ = run(w0, SeedHistory(K, N), gens)
+    w_half, hist = run(w0, SeedHistory(K, N), gens[:T // 2])
+    w_res, _ = run(np.frombuffer(w_half.tobytes(), np.uint8).copy(), SeedHistory.from_bytes(hist.to_bytes()), gens[T // 2:])
+    assert np.array_equal(w_full, w_res) and not np.array_equal(w_full, w0)
