@@ -519,3 +519,50 @@ def test_resume_from_weights_and_history_through_the_library(qo, qes):
     w_half, hist = run(w0, SeedHistory(K, N), gens[:T // 2])
     w_res, _ = run(np.frombuffer(w_half.tobytes(), np.uint8).copy(), SeedHistory.from_bytes(hist.to_bytes()), gens[T // 2:])
     assert np.array_equal(w_full, w_res) and not np.array_equal(w_full, w0)
+
+
+def test_random_configurations(qo, qes):
+    """Thirty seeded random small cases over every switch of the interface (bit width, ragged shapes, group
+    size, element offset, population, window, sigma incl. the 4-bit limit, both units, both boundary rules,
+    narrowed code ranges, antithetic pairs, both noise modes): update, history loop and perturbation."""
+    import torch
+    rng = np.random.default_rng(20260203)
+    total_near = 0
+    for case in range(30):
+        bits = int(rng.choice([4, 8]))
+        rows, cols = int(rng.integers(1, 40)), 32 * int(rng.integers(1, 24))
+        unit = int(rng.integers(0, 2))
+        group = int(rng.choice([g for g in (0, 32, 64, 128) if g == 0 or cols % g == 0])) if unit else 0
+        off = 32 * int(rng.integers(0, 1 << 20)) + (int(rng.integers(0, 4)) << 33)
+        anti = int(rng.integers(0, 2))
+        N = 2 * int(rng.integers(1, 9)) if anti else int(rng.integers(1, 17))
+        K = int(rng.integers(0, 6))
+        sigma = float(rng.choice([0.25, 0.5, 1.0, 2.5])) if not unit else float(rng.choice([0.006, 0.012, 0.03]))
+        lr = float(rng.choice([0.5, 1.0])) * (2.0 * sigma if unit else 1.0)
+        lim = 1 << (bits - 1)
+        qmin, qmax = (-lim, lim - 1) if rng.integers(0, 2) else (-(lim - 1) + int(rng.integers(0, 3)), lim - 1 - int(rng.integers(0, 3)))
+        kw = dict(sigma=sigma, lr=lr, gamma=float(rng.choice([0.0, 0.9, 1.0])), n_pop=N, sigma_unit=unit,
+                  boundary_mode=int(rng.integers(0, 2)), antithetic=anti, noise_mode=int(rng.integers(0, 2)))
+        to, tg, packed, scales = _case(qo, qes, bits, rows, cols, group=group, off=off, qmin=qmin, qmax=qmax, seed=case)
+        ho, hg = _hp(qo, qes, **kw)
+        sc_d, sc_o = (_dev(scales), scales) if unit else (None, None)
+        seeds = wl.draw_seeds(K + 1, N // 2 if anti else N, stream=1000 + case)
+        fit = wl.draw_fitness(K + 1, N, "student_t3" if case % 3 == 0 else "normal", stream=1000 + case)
+        what = f"case {case}: bits {bits} {rows}x{cols} g{group} N{N} K{K} {kw}"
+        w = _dev(packed)
+        qes.qes_update(tg, w, sc_d, _dev(seeds), _dev(fit), K, None, hg)
+        ref = qo.update(to, packed, sc_o, seeds, fit, K, ho)
+        total_near += _compare_update(qo, _host(w), bits, ref, what)
+        got = qo.unpack(bits, _host(w), rows * cols)
+        assert got.min() >= qmin and got.max() <= qmax, what
+        res = torch.empty(rows * cols, dtype=torch.float32, device="cuda")
+        qes.qes_replay_residual(tg, _dev(packed), sc_d, _dev(seeds[:K]), _dev(fit[:K]), K, hg, res)
+        rr = qo.replay_residual(to, packed, sc_o, seeds[:K], fit[:K], K, ho)
+        far = rr["band"] >= BAND
+        tol = TOL * max(1.0, float(np.abs(rr["e"]).max()))          # fp32 carries |u| up to a few units here
+        assert np.abs(_host(res).astype(np.float64) - rr["e"])[far].max(initial=0.0) <= tol, what
+        seed = int(seeds[-1, 0])
+        wp = _dev(np.zeros_like(packed))
+        qes.qes_perturb(tg, _dev(packed), wp, sc_d, seed, hg)
+        assert np.array_equal(_host(wp), qo.pack(bits, qo.perturb(to, packed, sc_o, seed, ho))), what
+    print(f"random configurations: {total_near} elements inside the rounding band")
