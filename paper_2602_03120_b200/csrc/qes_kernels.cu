@@ -174,8 +174,8 @@ __global__ void __launch_bounds__(kThreads) perturb_kernel(PassParams p, RoundKe
     if (PAIR) out_minus.store(p.w_out_minus, chunk);
 }
 
-// Expands the seeds of one generation into round keys, next to the fitness values (stored as
-// -F * 2^-24, the factor that turns the kernel's -delta * 2^24 back into F * delta) and the
+// Expands the seeds of one generation into round keys, next to the fitness values (stored as -F,
+// which turns the kernel's -delta back into F * delta) and the
 // seed's SeedConst for counter high word y_cta (the one almost every CTA has throughout).
 __device__ __noinline__ void stage_generation(uint32_t* buf, const uint64_t* seeds, const float* fitness, int n_seeds,
                                                  bool antithetic, uint32_t y_cta) {
@@ -191,7 +191,7 @@ __device__ __noinline__ void stage_generation(uint32_t* buf, const uint64_t* see
         d[2] = make_uint4(rk.a[8], rk.a[9], rk.b[0], rk.b[1]);
         d[3] = make_uint4(rk.b[2], rk.b[3], rk.b[4], rk.b[5]);
         d[4] = make_uint4(rk.b[6], rk.b[7], rk.b[8], rk.b[9]);
-        d[5] = make_uint4(__float_as_uint(F * -0x1p-24f), sc.hak, sc.la, sc.lak);   // pairs with -delta * 2^24
+        d[5] = make_uint4(__float_as_uint(-F), sc.hak, sc.la, sc.lak);   // pairs with -delta
     }
 }
 
@@ -265,7 +265,7 @@ __global__ void __launch_bounds__(kThreads, QES_MIN_BLOCKS) pass_kernel(PassPara
         for (int t = 0; t < T; ++t) S[t] = 0.0f;
 #pragma unroll 1
         for (int i = 0; i < p.n_seeds; ++i) {
-            float Fm;   // -F_i * 2^-24
+            float Fm;   // -F_i
             SeedConst sc;
             const RoundKeys rk = load_round_keys(table + i * kSeedStride, Fm, sc);
             if (!y_uniform) sc = make_seed_const(y, rk);
@@ -277,7 +277,7 @@ __global__ void __launch_bounds__(kThreads, QES_MIN_BLOCKS) pass_kernel(PassPara
                 call_rounding_sums<CLAMP_DELTA, QUAD>(r0, r1, r2, r3, nsig24, z);
 #pragma unroll
                 for (int j = 0; j < kPerCall; ++j)          // Eq. 5 numerator
-                    S[kPerCall * c + j] = fmaf(Fm, neg_delta_scaled<CLAMP_DELTA>(z[j], p.nd_max), S[kPerCall * c + j]);
+                    S[kPerCall * c + j] = fmaf(Fm, neg_delta_float<CLAMP_DELTA>(z[j], p.nd_max), S[kPerCall * c + j]);
             }
         }
         const bool is_update = (k == last) && (p.mode != kReplayOnly);
