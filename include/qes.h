@@ -140,7 +140,8 @@ int qes_update(const qes_tensor_desc* desc, void* w_inout, const void* scales_f1
  * names no generator, this library fixes one): for each i, radius[i] = sqrt(-2 ln u1) with
  * u1 = ((r0[i] >> 8) + 1) / 2^24, and (cosine[i], sine[i]) of 2*pi*u2 with u2 = (r1[i] >> 8) / 2^24,
  * each by the library's fixed fp32 operation sequence.  Lets a caller check that sequence on its
- * whole domain (2^24 values per factor).  All five arrays are DEVICE pointers to n elements,
+ * whole domain (2^24 values per factor).  The kernels use two forms of the square root; where they
+ * disagree radius[i] is NaN.  All five arrays are DEVICE pointers to n elements,
  * owned by the caller; n == 0 is a no-op.  Enqueues on cuda_stream, does not synchronise.
  */
 int qes_gaussian_factors(const uint32_t* r0, const uint32_t* r1, int64_t n, float* radius, float* cosine,

@@ -326,7 +326,9 @@ __global__ void __launch_bounds__(kThreads) gaussian_factors_kernel(const uint32
                                                                     float* R, float* C, float* S) {
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
-    R[i] = bm_radius(r0[i]);
+    // the two square-root forms the kernels use must agree; a disagreement shows as NaN
+    const float ra = bm_radius<false>(r0[i]), rb = bm_radius<true>(r0[i]);
+    R[i] = ra == rb ? ra : __uint_as_float(0x7fc00000u);
     float c, s;
     bm_cossin(r1[i], c, s);
     C[i] = c;
