@@ -1,6 +1,6 @@
 """Parity of the CUDA library (through its C ABI) against the CPU oracle, element by element.
 
-Rules (the benchmark spec): packed codes bit-exact, except elements whose pre-rounding value u lies within
+Rules: packed codes bit-exact, except elements whose pre-rounding value u lies within
 1e-5 of a rounding boundary in any generation (counted, reported, never silently skipped);
 residuals within 1e-5 absolute on the remaining elements.  qes_perturb has no such band: exact.
 """
