@@ -269,11 +269,8 @@ def main():
         barrier()
         a, b = ev(), ev(); a.record(stream)
         for _ in range(e2e_steps):
-            model.load(host)
             s_d, f_d = seeds_h.cuda(non_blocking=True), fit_h.cuda(non_blocking=True)
-            perturb_all()
-            model.update(s_d, f_d, cfg.K)
-            host_out.copy_(model.w, non_blocking=True)
+            model.step_from_host(host, host_out, scratch, member_seeds, s_d, f_d, cfg.K, scratch_minus)
         b.record(stream)
         barrier()
         e_ms = a.elapsed_time(b) / e2e_steps

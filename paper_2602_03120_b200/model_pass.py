@@ -120,3 +120,38 @@ class ModelPass:
             lo = t.elem_offset - self.base
             qes.qes_replay_residual(d, self._slice(self.w, t), sc, seeds, fitness, K, self.hp, out[lo:lo + t.numel])
         return len(calls)
+
+    def step_from_host(self, host_in: torch.Tensor, host_out: torch.Tensor, scratch: torch.Tensor, member_seeds,
+                       seeds: torch.Tensor, fitness: torch.Tensor, K: int, scratch_minus: torch.Tensor | None = None) -> int:
+        """One full step (the perturbation of every member, then the stateless update) with the weights
+        starting and ending in pinned host memory.  The set is walked launch by launch: the copy-in of
+        the next run of tensors and the copy-out of the previous one ride on two side streams under the
+        arithmetic of the current one, so only the first copy-in and the last copy-out are exposed."""
+        main = torch.cuda.current_stream()
+        if not hasattr(self, "_copy_in"):
+            self._copy_in, self._copy_out = torch.cuda.Stream(), torch.cuda.Stream()
+        calls = self._launches()
+        self._copy_in.wait_stream(main)          # the previous step's kernels are done with self.w
+        self._copy_out.wait_stream(main)
+        arrived = []
+        for t, _, _ in calls:
+            with torch.cuda.stream(self._copy_in):
+                self._slice(self.w, t).copy_(self._slice(host_in, t), non_blocking=True)
+                ev = torch.cuda.Event(); ev.record(self._copy_in); arrived.append(ev)
+        n = 0
+        for (t, d, sc), ev in zip(calls, arrived):
+            main.wait_event(ev)
+            w_t = self._slice(self.w, t)
+            for s in member_seeds:                                   # Algorithm 1, member loop
+                if scratch_minus is not None:
+                    qes.qes_perturb_pair(d, w_t, self._slice(scratch, t), self._slice(scratch_minus, t), sc, s, self.hp)
+                else:
+                    qes.qes_perturb(d, w_t, self._slice(scratch, t), sc, s, self.hp)
+            qes.qes_update(d, w_t, sc, seeds, fitness, K, None, self.hp)     # Algorithm 2
+            n += len(member_seeds) + 1
+            done = torch.cuda.Event(); done.record(main)
+            with torch.cuda.stream(self._copy_out):
+                self._copy_out.wait_event(done)
+                self._slice(host_out, t).copy_(w_t, non_blocking=True)
+        main.wait_stream(self._copy_out)         # the step ends when the last bytes are back on the host
+        return n

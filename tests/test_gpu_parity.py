@@ -566,3 +566,44 @@ def test_random_configurations(qo, qes):
         qes.qes_perturb(tg, _dev(packed), wp, sc_d, seed, hg)
         assert np.array_equal(_host(wp), qo.pack(bits, qo.perturb(to, packed, sc_o, seed, ho))), what
     print(f"random configurations: {total_near} elements inside the rounding band")
+
+
+def test_step_from_host_equals_the_resident_step(qo, qes):
+    """The end-to-end call (weights in pinned host memory, copies pipelined under the arithmetic on side
+    streams) gives the bytes of the resident path, twice in a row, and leaves the last member's perturbation
+    in the scratch copy."""
+    import torch
+    from paper_2602_03120_b200.model_pass import ModelPass, MAX_SEGMENT_ELEMS
+    cfg = wl.WORKLOADS["decoder1p5b_int4"]
+    tensors = cfg.tensors[:14]                                   # two layers, 93.6M codes
+    seeds, fit = wl.draw_seeds(cfg.K + 1, cfg.n_pop), wl.draw_fitness(cfg.K + 1, cfg.n_pop)
+    member_seeds = [int(s) for s in seeds[-1][:3]]
+    import paper_2602_03120_b200.model_pass as mp
+    old = mp.MAX_SEGMENT_ELEMS
+    mp.MAX_SEGMENT_ELEMS = 1 << 25                               # several launches, so the pipeline has stages
+    try:
+        model = ModelPass(cfg, tensors=tensors)
+        segs = mp.launch_segments(tensors, mp.MAX_SEGMENT_ELEMS)
+        model.segments = [(wl.TensorSpec(f"segment{j}", n // 32, 32, off),
+                           qes.TensorDesc(bits=4, rows=n // 32, cols=32, elem_offset=off)) for j, (_, off, n) in enumerate(segs)]
+        assert len(model.segments) >= 3
+    finally:
+        mp.MAX_SEGMENT_ELEMS = old
+    host = torch.from_numpy(model.host_codes()).pin_memory()
+    out = torch.empty_like(host).pin_memory()
+    scratch = torch.empty_like(model.w)
+    ds, df = _dev(seeds), _dev(fit)
+    model.load(host)
+    model.update(ds, df, cfg.K)
+    want = _host(model.w)
+    want_scratch = torch.empty_like(model.w)
+    model.load(host)
+    model.perturb_member(want_scratch, member_seeds[-1])
+    for _ in range(2):
+        out.zero_()
+        n = model.step_from_host(host, out, scratch, member_seeds, ds, df, cfg.K)
+        torch.cuda.synchronize()
+        assert n == len(model.segments) * (len(member_seeds) + 1)
+        assert np.array_equal(out.numpy(), want)
+        assert torch.equal(scratch, want_scratch)
+    assert not np.array_equal(want, host.numpy())
