@@ -1,19 +1,21 @@
 // Kernels and C ABI of the QES parameter pass (sm_100a).  See include/qes.h for the contract.
 //
-// Work decomposition: one thread owns 2*kPairs consecutive codes (kPairs Philox calls per seed).
-// With kPairs = 4 that is one 32-bit load for INT4 and one 64-bit load for INT8: a warp reads and
-// writes one contiguous 128 B / 256 B segment, once.  Everything else is arithmetic in
-// registers: a code costs one byte of HBM traffic but N*(K+1) noise samples of ~50 operations
-// each, so the kernels are bound by instruction issue on the multiply and integer pipes, never
-// by memory; kPairs is chosen for the register budget (S, e and the Philox state of 4 pairs fit
-// without spills at two CTAs per SM), not for the width of the load.
+// Work decomposition: one thread owns 2*kPairs consecutive codes: kPairs Philox calls per seed
+// in the default noise mode, half as many when one call serves four elements.  With kPairs = 4
+// that is one 32-bit load for INT4 and one 64-bit load for INT8: a warp reads and writes one
+// contiguous 128 B / 256 B segment, once.  Everything else is arithmetic in registers: a code
+// costs one byte of HBM traffic but N*(K+1) noise samples of ~50 operations each, so the
+// kernels are bound by instruction issue on the multiply and integer pipes, never by memory;
+// kPairs is chosen for the register budget (S, e and the Philox state of 4 pairs fit without
+// spills at two CTAs per SM), not for the width of the load.
 //
-// Per generation the CTA stages, in shared memory, the ten Philox round keys of each of the N
-// seeds next to the member's fitness (96 B per member, double-buffered so one barrier per
-// generation suffices); every thread then walks the members in the same order, each table read
-// is a broadcast, and a seed's keys are fetched with five 128-bit loads instead of being
-// re-derived by 18 additions per thread.  The residual e and the weighted sums S of Eqs. 5-8
-// never leave registers between generations (Algorithm 2 keeps no O(d) state).
+// Per generation the CTA stages, in shared memory, the ten Philox round keys of each seed next
+// to the member's fitness and the seed's share of the first Philox rounds (96 B per seed,
+// double-buffered so one barrier per generation suffices); every thread then walks the seeds in
+// the same order, each table read is a broadcast, and a seed's entry is fetched with six
+// 128-bit loads instead of being re-derived by 18 additions and a wide multiply per thread.
+// The residual e and the weighted sums S of Eqs. 5-8 never leave registers between generations
+// (Algorithm 2 keeps no O(d) state).
 #include "qes_device.cuh"
 #include "../../include/qes.h"
 
