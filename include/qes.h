@@ -161,6 +161,7 @@ int qes_gaussian_factors(const uint32_t* r0, const uint32_t* r1, int64_t n, floa
  *         per step)  20/21/22 the same plus 1/2/4 independent fp32 fma per step
  *         23/24/25 the update kernel's mix per step (one wide multiply, 2.5 xor3, 2 fp32 fma) in three
  *         program orders: chain by chain, kinds alternating, kinds grouped
+ *         26 fma.rn.f32x2 (packed pair of fp32 fma, counted per instruction)  27 mul.wide.u32 + xor3 + one f32x2 per step
  *         100-109 two-kind mixes (see the binding's PROBE_KINDS)
  */
 int qes_pipe_probe(int32_t kind, int32_t iters, void* sink_dev, float* ms_out, double* ops_out);

@@ -225,6 +225,7 @@ PROBE_KINDS = {0: "mul.wide.u32", 1: "lop3.xor3", 2: "fma.rn.f32", 3: "mul.hi.u3
                21: "mul.wide + xor3 + 2 fma (steps)", 22: "mul.wide + xor3 + 4 fma (steps)",
                23: "update-kernel mix: wide + 2.5 xor3 + 2 fma (steps)",
                24: "the same mix, kinds alternating (steps)", 25: "the same mix, kinds grouped (steps)",
+               26: "fma.rn.f32x2 (instructions, two fmas each)", 27: "mul.wide + xor3 + 1 fma.f32x2 (steps)",
                100: "mix mul.wide + xor3", 101: "mix fma + xor3", 102: "mix mul.wide + fma", 103: "mix cvt.f32.u32 + xor3",
                104: "mix cvt.f32.u32 + mul.wide", 105: "mix floor + rsqrt", 106: "mix floor + fma", 107: "mix add + xor3",
                108: "mix fadd + mul.wide", 109: "mix setp/selp + fma"}

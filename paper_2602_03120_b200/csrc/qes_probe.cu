@@ -167,6 +167,61 @@ __global__ void __launch_bounds__(kProbeThreads) probe_wide_kernel(int iters, ui
     if (acc == 0x12345u) sink[0] = acc;
 }
 
+// Packed fp32: fma.rn.f32x2 does two fused multiply-adds per instruction on a 64-bit register
+// pair.  WITH_WIDE == false: a pure chain (instructions per second); true: one wide multiply +
+// xor3 + one f32x2 per step, to compare with the same step carrying two scalar fmas.
+template <bool WITH_WIDE>
+__global__ void __launch_bounds__(kProbeThreads) probe_f32x2_kernel(int iters, uint32_t a, uint32_t b, uint32_t* sink) {
+    unsigned long long f[kChains], w[kChains];
+    const float fa = __uint_as_float(b), fb = 1e-7f;
+    unsigned long long aa, bb;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(aa) : "f"(fa), "f"(fa));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(bb) : "f"(fb), "f"(fb));
+#pragma unroll
+    for (int c = 0; c < kChains; ++c) {
+        float x = 1.0f + 1e-3f * (float)(threadIdx.x + c), y = 1.0f - 1e-3f * (float)c;
+        asm("mov.b64 %0, {%1, %2};" : "=l"(f[c]) : "f"(x), "f"(y));
+        w[c] = ((unsigned long long)(threadIdx.x * 2654435761u + c * 40503u) << 32) | (blockIdx.x + 0x3f800001u + c);
+    }
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int c = 0; c < kChains; ++c) {
+            if (WITH_WIDE) {
+                unsigned long long p;
+                asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(p) : "r"((uint32_t)w[c]), "r"(a));
+                w[c] = (uint32_t)(p >> 32) ^ (uint32_t)p ^ b;
+            }
+            asm volatile("fma.rn.f32x2 %0, %0, %1, %2;" : "+l"(f[c]) : "l"(aa), "l"(bb));
+        }
+    }
+    uint32_t acc = 0;
+#pragma unroll
+    for (int c = 0; c < kChains; ++c) acc ^= (uint32_t)f[c] ^ (uint32_t)(f[c] >> 32) ^ (uint32_t)w[c];
+    if (acc == 0x12345u) sink[0] = acc;
+}
+
+template <bool WITH_WIDE>
+int run_f32x2(int iters, uint32_t* sink, float* ms_out, double* ops_out) {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return QES_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return QES_ERR_CUDA;
+    cudaEvent_t e0, e1;
+    cudaEventCreate(&e0); cudaEventCreate(&e1);
+    int blocks = sms * kCtasPerSm;
+    probe_f32x2_kernel<WITH_WIDE><<<blocks, kProbeThreads>>>(iters / 8 + 1, 0xD2511F53u, 0x3f7ffff0u, sink);
+    cudaEventRecord(e0);
+    probe_f32x2_kernel<WITH_WIDE><<<blocks, kProbeThreads>>>(iters, 0xD2511F53u, 0x3f7ffff0u, sink);
+    cudaEventRecord(e1);
+    cudaError_t err = cudaEventSynchronize(e1);
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, e0, e1);
+    cudaEventDestroy(e0); cudaEventDestroy(e1);
+    if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return QES_ERR_CUDA;
+    *ms_out = ms;
+    *ops_out = (double)blocks * kProbeThreads * (double)iters * (double)kChains;   // f32x2 instructions, or steps
+    return QES_OK;
+}
+
 // The instruction mix of the update kernel with full instruction-level parallelism: per step
 // one wide multiply, 2.5 half-rate integer operations (the xor3 of the products plus 1.5
 // independent xor3) and two independent fp32 fused multiply-adds -- by the pipe rates 6 cycles
@@ -373,6 +428,8 @@ extern "C" int qes_pipe_probe(int32_t kind, int32_t iters, void* sink_dev, float
         case 23: return run_mix_pass<0>(iters, sink, ms_out, ops_out);
         case 24: return run_mix_pass<1>(iters, sink, ms_out, ops_out);
         case 25: return run_mix_pass<2>(iters, sink, ms_out, ops_out);
+        case 26: return run_f32x2<false>(iters, sink, ms_out, ops_out);
+        case 27: return run_f32x2<true>(iters, sink, ms_out, ops_out);
         case 100: return run_mix<0, 1>(iters, sink, ms_out, ops_out);    // mul.wide + xor3
         case 101: return run_mix<2, 1>(iters, sink, ms_out, ops_out);    // fma + xor3
         case 102: return run_mix<0, 2>(iters, sink, ms_out, ops_out);    // mul.wide + fma
