@@ -1,9 +1,10 @@
 /*
  * libqes — the per-iteration parameter pass of Quantized Evolution Strategies (QES) on one GPU.
  *
- * Three operations over a packed low-bit weight tensor, every noise sample regenerated in
+ * The operations over a packed low-bit weight tensor, every noise sample regenerated in
  * registers from integer seeds (nothing but the weights is ever stored):
  *   qes_perturb          W' = Gate(W + delta_i)                     Algorithm 1, member loop; Eqs. 3-4
+ *   qes_perturb_pair     both members W +- delta of an antithetic pair  App. A
  *   qes_update           reward-weighted sum, error feedback, round,
  *                        gate, repack — with Stateless Seed Replay     Algorithm 2; Eqs. 5-8
  *                        or with a stored residual                     Algorithm 1, update lines
@@ -20,8 +21,8 @@
  *  - Scales: IEEE binary16, [rows, cols / group_size] row-major, or [rows] when group_size == 0.
  *    Read only when sigma_unit == QES_SIGMA_WEIGHT; may be NULL otherwise.
  *  - Noise: delta(seed, J) for global element index J = elem_offset + row*cols + col is
- *    Philox4x32-10(key = seed, counter = J >> 1) -> Box-Muller -> sigma scaling -> stochastic
- *    rounding (Eq. 3), limited to the 4-bit range [-8, 7] (App. A).  Results depend only on
+ *    Philox4x32-10(key = seed, counter = J >> 1, or J >> 2 in the QES_NOISE_QUAD8 mode) -> Box-Muller ->
+ *    sigma scaling -> stochastic rounding (Eq. 3), limited to the 4-bit range [-8, 7] (App. A).  Results depend only on
  *    (seed, J): any split of a model into tensors, any grid size, gives the same bits.
  *    With sigma_unit == QES_SIGMA_WEIGHT, sigma / scale above 2^40 is treated as 2^40 (every
  *    non-zero sample saturates the 4-bit range long before).
@@ -45,9 +46,9 @@ typedef enum {
     QES_ERR_BAD_SHAPE = -3,   /* rows/cols/group_size/elem_offset violate the layout rules */
     QES_ERR_MISALIGNED = -4,  /* a device pointer misses its alignment (16 B weights/residual, 8 B seeds, 4 B fitness, 2 B scales) */
     QES_ERR_BAD_HPARAM = -5,  /* sigma <= 0, n_pop <= 0 (or odd with antithetic pairs), K < 0, gamma outside [0,1], qmin >= qmax, range outside the code width */
-    QES_ERR_BAD_MODE = -6,    /* unknown sigma_unit / boundary_mode / antithetic, residual_inout given with K > 0, qes_perturb_pair without antithetic, or its two outputs the same buffer */
+    QES_ERR_BAD_MODE = -6,    /* unknown sigma_unit / boundary_mode / antithetic / residual_f16 / noise_mode, residual_inout given with K > 0, qes_perturb_pair without antithetic, or its two outputs the same buffer */
     QES_ERR_CUDA = -7,        /* the launch reported a CUDA error (cudaGetLastError) */
-    QES_ERR_TOO_LARGE = -8    /* n_pop exceeds what one generation's shared-memory staging holds (1066 members) */
+    QES_ERR_TOO_LARGE = -8    /* more seeds per generation than the shared-memory staging holds (1066: members, or antithetic pairs) */
 } qes_status;
 
 enum { QES_SIGMA_GRID = 0, QES_SIGMA_WEIGHT = 1 };   /* unit of hparams.sigma: grid steps | weight units (sigma_g = sigma / scale_g) */
