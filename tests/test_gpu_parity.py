@@ -261,36 +261,39 @@ def test_gaussian_factors_bit_identical_on_the_whole_domain(qo, qes):
             f"{name}: {(g.view(np.uint32) != want.view(np.uint32)).sum()} of 2^24 values differ"
 
 
-def test_fused_launch_segments_match_per_tensor_oracle(qo, qes):
+@pytest.mark.parametrize("name,n_tensors,n_segments", [("decoder7b_int4", 14, 2), ("decoder7b_int8", 7, 1),
+                                                       ("decoder8b_int4", 3, 1)])
+def test_fused_launch_segments_match_per_tensor_oracle(qo, qes, name, n_tensors, n_segments):
     """The whole-model pass the benchmark times: runs of consecutive tensors go to the library as one
-    [numel / 32, 32] tensor (at most 2^28 codes per call).  Checked on the first two layers of the 7B-shaped
-    INT4 set (14 tensors, two segments) against the oracle run tensor by tensor with each tensor's own
-    geometry, on sampled words that include both ends of every tensor."""
+    [numel / 32, 32] tensor (at most 2^28 codes per call).  Checked on the leading tensors of the 7B-shaped INT4
+    and INT8 sets and of the 8B-shaped set (N = 64, K = 64) against the oracle run tensor by tensor with each
+    tensor's own geometry, on sampled words that include both ends of every tensor."""
     from paper_2602_03120_b200.model_pass import ModelPass, launch_segments
-    cfg = wl.WORKLOADS["decoder7b_int4"]
-    tensors = cfg.tensors[:14]
+    cfg = wl.WORKLOADS[name]
+    tensors = cfg.tensors[:n_tensors]
     model = ModelPass(cfg, tensors=tensors)
-    assert len(model.segments) == len(launch_segments(tensors)) == 2
+    assert len(model.segments) == len(launch_segments(tensors)) == n_segments
     assert sum(t.numel for t, _ in model.segments) == sum(t.numel for t in tensors)
     host = model.host_codes()
     model.load(host)
     seeds, fit = wl.draw_seeds(cfg.K + 1, cfg.n_pop), wl.draw_fitness(cfg.K + 1, cfg.n_pop, cfg.reward_dist)
-    assert model.update(_dev(seeds), _dev(fit), cfg.K) == 2
+    assert model.update(_dev(seeds), _dev(fit), cfg.K) == n_segments
     got_all = _host(model.w)
     ho = qo.HParams(sigma=cfg.sigma, lr=cfg.lr, gamma=cfg.gamma, n_pop=cfg.n_pop)
+    per_tensor = 512 if cfg.K <= 16 else 128
     near_total = 0
     for ti, t in enumerate(tensors):
-        lo = t.elem_offset // 2
-        packed = host[lo:lo + t.numel // 2]
+        lo, nb = wl.packed_bytes(cfg.bits, t.elem_offset), wl.packed_bytes(cfg.bits, t.numel)
+        packed = host[lo:lo + nb]
         assert np.array_equal(packed, wl.draw_codes(cfg, ti))
-        to = qo.Tensor(bits=4, rows=t.rows, cols=t.cols, group_size=cfg.group_size, elem_offset=t.elem_offset)
-        idx = wl.sample_elements(t.numel, 512, stream=100 + ti)
+        to = qo.Tensor(bits=cfg.bits, rows=t.rows, cols=t.cols, group_size=cfg.group_size, elem_offset=t.elem_offset)
+        idx = wl.sample_elements(t.numel, per_tensor, stream=100 + ti)
         ref = qo.update(to, packed, None, seeds, fit, cfg.K, ho, idx=idx)
-        got = qo.unpack(4, got_all[lo:lo + t.numel // 2], t.numel)[idx]
+        got = qo.unpack(cfg.bits, got_all[lo:lo + nb], t.numel)[idx]
         near = ref["band"] < BAND
         assert not np.any((got != ref["w_new"]) & ~near), f"tensor {ti} ({t.name})"
         near_total += int(near.sum())
-    print(f"fused segments: near-band sampled elements {near_total}")
+    print(f"fused segments ({name}): near-band sampled elements {near_total}")
 
 
 @pytest.mark.parametrize("bits,off", [(4, (1 << 33) - 1024), (8, (1 << 33) - 32), (4, (1 << 33) - 2048)])
