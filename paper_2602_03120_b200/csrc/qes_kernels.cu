@@ -133,17 +133,18 @@ __device__ __forceinline__ float applied_step(float w, float step, float qmin, f
     return fminf(fmaxf(target, qmin), qmax) - w;
 }
 
-// The same rule on integer codes: the code after the step.
-__device__ __forceinline__ int applied_code(int w, int step, int qmin, int qmax, int boundary_mode) {
+// The same rule on integer codes: the code after the step (one unsigned comparison for the gate).
+template <bool CLAMP_CODE>
+__device__ __forceinline__ int applied_code(int w, int step, int qmin, int qmax) {
     int target = w + step;
-    if (boundary_mode == QES_BOUNDARY_GATE) return (target >= qmin && target <= qmax) ? target : w;
-    return min(max(target, qmin), qmax);
+    if (CLAMP_CODE) return min(max(target, qmin), qmax);
+    return (unsigned)(target - qmin) <= (unsigned)(qmax - qmin) ? target : w;
 }
 
 // Algorithm 1, member loop: W' = Gate(W + delta_i), and with PAIR also the antithetic member
 // Gate(W - delta_i) from the same noise.  The member's round keys are computed on the host and
 // arrive as kernel parameters, i.e. as constant-bank operands.
-template <int BITS, bool CLAMP_DELTA, bool PAIR, bool QUAD>
+template <int BITS, bool CLAMP_DELTA, bool PAIR, bool QUAD, bool CLAMP_CODE>
 __global__ void __launch_bounds__(kThreads) perturb_kernel(PassParams p, RoundKeys rk) {
     constexpr int kPerCall = QUAD ? 4 : 2;                 // elements served by one Philox call
     constexpr int kCalls = kCodesPerThread / kPerCall;
@@ -168,8 +169,8 @@ __global__ void __launch_bounds__(kThreads) perturb_kernel(PassParams p, RoundKe
         for (int j = 0; j < kPerCall; ++j) {
             const int t = kPerCall * i + j;
             const int nd = neg_delta<CLAMP_DELTA>(z[j], p.nd_max), wc = w.get(t);
-            out.put(t, applied_code(wc, -nd, p.qmin_i, p.qmax_i, p.boundary_mode));
-            if (PAIR) out_minus.put(t, applied_code(wc, nd, p.qmin_i, p.qmax_i, p.boundary_mode));
+            out.put(t, applied_code<CLAMP_CODE>(wc, -nd, p.qmin_i, p.qmax_i));
+            if (PAIR) out_minus.put(t, applied_code<CLAMP_CODE>(wc, nd, p.qmin_i, p.qmax_i));
         }
     }
     out.store(p.w_out, chunk);
@@ -429,15 +430,21 @@ int check_table(const uint64_t* seeds, const float* fitness, int64_t generations
     return QES_OK;
 }
 
+template <int BITS, bool QUAD, bool CLAMP_CODE>
+void launch_perturb_mode(bool clamp, bool pair, const PassParams& p, const RoundKeys& rk, unsigned blocks, cudaStream_t stream) {
+    if (clamp) {
+        if (pair) perturb_kernel<BITS, true, true, QUAD, CLAMP_CODE><<<blocks, kThreads, 0, stream>>>(p, rk);
+        else perturb_kernel<BITS, true, false, QUAD, CLAMP_CODE><<<blocks, kThreads, 0, stream>>>(p, rk);
+    } else {
+        if (pair) perturb_kernel<BITS, false, true, QUAD, CLAMP_CODE><<<blocks, kThreads, 0, stream>>>(p, rk);
+        else perturb_kernel<BITS, false, false, QUAD, CLAMP_CODE><<<blocks, kThreads, 0, stream>>>(p, rk);
+    }
+}
+
 template <int BITS, bool QUAD>
 void launch_perturb_bits(bool clamp, bool pair, const PassParams& p, const RoundKeys& rk, unsigned blocks, cudaStream_t stream) {
-    if (clamp) {
-        if (pair) perturb_kernel<BITS, true, true, QUAD><<<blocks, kThreads, 0, stream>>>(p, rk);
-        else perturb_kernel<BITS, true, false, QUAD><<<blocks, kThreads, 0, stream>>>(p, rk);
-    } else {
-        if (pair) perturb_kernel<BITS, false, true, QUAD><<<blocks, kThreads, 0, stream>>>(p, rk);
-        else perturb_kernel<BITS, false, false, QUAD><<<blocks, kThreads, 0, stream>>>(p, rk);
-    }
+    if (p.boundary_mode == QES_BOUNDARY_CLAMP) launch_perturb_mode<BITS, QUAD, true>(clamp, pair, p, rk, blocks, stream);
+    else launch_perturb_mode<BITS, QUAD, false>(clamp, pair, p, rk, blocks, stream);
 }
 
 // w_minus == nullptr: one member; otherwise both members of an antithetic pair.
