@@ -202,7 +202,7 @@ def test_config1_full_matrix(qo, qes):
     assert (ref["w_new"] != qo.unpack(4, packed, t.numel)).mean() > 0.01
 
 
-@pytest.mark.parametrize("name", ["decoder7b_int4", "decoder7b_int8", "decoder8b_int4"])
+@pytest.mark.parametrize("name", ["decoder1p5b_int4", "decoder7b_int4", "decoder7b_int8", "decoder8b_int4"])
 def test_full_size_tensors_sampled(qo, qes, name):
     """Full-size tensors of the large configurations in the benchmark's launch configuration (one call per
     tensor, the configuration's N and K), oracle on sampled 32-element words incl. first and last."""
