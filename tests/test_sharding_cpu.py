@@ -63,3 +63,32 @@ def test_shard_of_a_deeper_model_equals_that_slice_of_it(qo):
     part = qo.update(qo.Tensor(bits=4, rows=n // 32, cols=32, elem_offset=t1.elem_offset), packed, None, seeds, fit, 2, hp)
     assert np.array_equal(whole["w_new"][n:], part["w_new"])
     assert not np.array_equal(whole["w_new"][:n], part["w_new"])
+
+
+def test_launch_segments_cover_every_tensor_once_and_respect_the_limit():
+    """Runs of consecutive tensors for the fused launches: contiguous, in order, no run above the limit
+    unless a single tensor is, and a gap in the element offsets starts a new run."""
+    from paper_2602_03120_b200.model_pass import launch_segments
+    rng = np.random.default_rng(4)
+    for trial in range(50):
+        sizes = (32 * rng.integers(1, 400, size=int(rng.integers(1, 30)))).tolist()
+        gaps = set(rng.integers(0, len(sizes), size=2).tolist()) if trial % 3 == 0 else set()
+        tensors, off = [], 0
+        for i, n in enumerate(sizes):
+            if i in gaps and i > 0:
+                off += 64
+            tensors.append(wl.TensorSpec(f"t{i}", n // 32, 32, off)); off += n
+        limit = int(32 * rng.integers(1, 600))
+        segs = launch_segments(tensors, limit)
+        covered = []
+        for first, seg_off, n in segs:
+            assert tensors[first].elem_offset == seg_off
+            run, j = 0, first
+            while run < n:
+                assert tensors[j].elem_offset == seg_off + run      # contiguous inside a run
+                run += tensors[j].numel; covered.append(j); j += 1
+            assert run == n
+            assert n <= limit or j == first + 1                       # only a lone tensor may exceed the limit
+        assert covered == list(range(len(tensors)))
+    cfg = wl.WORKLOADS["decoder7b_int4"]
+    assert len(launch_segments(cfg.tensors)) == 28 and max(s[2] for s in launch_segments(cfg.tensors)) <= 1 << 28
