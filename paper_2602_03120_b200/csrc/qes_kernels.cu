@@ -213,7 +213,7 @@ __device__ __forceinline__ RoundKeys load_round_keys(const uint32_t* entry, floa
 }
 
 // Algorithm 2 (stateless), Algorithm 1's update lines (stored residual) or the history loop
-// alone (replay only), selected by p.mode.  Shared memory: 2 * n_pop * 96 B.
+// alone (replay only), selected by p.mode.  Shared memory: 2 * (seeds per generation) * 96 B.
 template <int BITS, bool CLAMP_DELTA, bool STATS, bool QUAD>
 __global__ void __launch_bounds__(kThreads, QES_MIN_BLOCKS) pass_kernel(PassParams p) {
     extern __shared__ __align__(16) uint32_t smem[];
