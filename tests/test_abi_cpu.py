@@ -83,3 +83,38 @@ def test_binding_refuses_host_tensors():
     w = torch.zeros(128, dtype=torch.uint8)
     with pytest.raises(binding.QesError):
         binding.qes_perturb(d, w, w, None, 1, h, stream=0)
+
+
+def test_header_is_plain_c_and_links_from_a_c_program(tmp_path, lib):
+    """include/qes.h compiles as C99 on its own, and a C program linked against the library gets the
+    documented status codes for invalid arguments (no device needed: validation precedes any CUDA call)."""
+    import subprocess
+    from paper_2602_03120_b200 import binding
+    header = os.path.join(ROOT, "include", "qes.h")
+    subprocess.run(["gcc", "-x", "c", "-std=c99", "-Wall", "-Wextra", "-Werror", "-fsyntax-only", header], check=True)
+    src = tmp_path / "abi.c"
+    src.write_text(r'''
+#include <stdio.h>
+#include <string.h>
+#include "qes.h"
+int main(void) {
+    qes_tensor_desc d; qes_hparams h;
+    memset(&d, 0, sizeof d); memset(&h, 0, sizeof h);
+    d.bits = 4; d.qmin = -8; d.qmax = 7; d.rows = 4; d.cols = 64;
+    h.sigma = 0.5f; h.lr = 1.0f; h.gamma = 0.9f; h.n_pop = 4;
+    int a = qes_update(NULL, (void*)0x1000, NULL, (const uint64_t*)0x2000, (const float*)0x3000, 1, NULL, &h, NULL, NULL);
+    d.bits = 5;
+    int b = qes_update(&d, (void*)0x1000, NULL, (const uint64_t*)0x2000, (const float*)0x3000, 1, NULL, &h, NULL, NULL);
+    d.bits = 4; d.cols = 48;
+    int c = qes_perturb(&d, (const void*)0x1000, (void*)0x1000, NULL, 1, &h, NULL);
+    printf("%d %d %d %d %s\n", qes_version(), a, b, c, qes_strerror(c));
+    return 0;
+}
+''')
+    exe = tmp_path / "abi"
+    libdir = os.path.dirname(binding.LIB_PATH)
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", f"-I{os.path.join(ROOT, 'include')}", str(src), "-o", str(exe),
+                    f"-L{libdir}", "-l:libqes.so", f"-Wl,-rpath,{libdir}"], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split(maxsplit=4)
+    assert int(out[0]) >= 100 and [int(v) for v in out[1:4]] == [-1, -2, -3]
+    assert "layout" in out[4]
