@@ -610,3 +610,23 @@ def test_step_from_host_equals_the_resident_step(qo, qes):
         assert np.array_equal(out.numpy(), want)
         assert torch.equal(scratch, want_scratch)
     assert not np.array_equal(want, host.numpy())
+
+
+def test_calls_run_on_the_callers_stream(qo, qes):
+    """The library enqueues on the stream it is given and never synchronises: two updates issued on two side
+    streams (one passed explicitly, one as torch's current stream) give the default-stream result."""
+    import torch
+    to, tg, packed, _ = _case(qo, qes, 4, 64, 512, off=128)
+    _, hg = _hp(qo, qes, sigma=0.5, lr=1.0, gamma=0.9, n_pop=8)
+    seeds, fit = _dev(wl.draw_seeds(4, 8, stream=7)), _dev(wl.draw_fitness(4, 8, stream=7))
+    want = _dev(packed)
+    qes.qes_update(tg, want, None, seeds, fit, 3, None, hg)
+    torch.cuda.synchronize()
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    a, b = _dev(packed), _dev(packed)
+    torch.cuda.synchronize()
+    qes.qes_update(tg, a, None, seeds, fit, 3, None, hg, stream=s1)
+    with torch.cuda.stream(s2):
+        qes.qes_update(tg, b, None, seeds, fit, 3, None, hg)
+    s1.synchronize(); s2.synchronize()
+    assert torch.equal(a, want) and torch.equal(b, want)
