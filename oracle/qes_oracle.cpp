@@ -112,8 +112,9 @@ int stochastic_round_exact(float x, double v, int dmin) {
     double xd = (double)x;
     double fl = std::floor(xd);
     double frac = xd - fl;                          // exact
-    int d = (int)fl + (v < frac ? 1 : 0);
-    return std::min(7, std::max(dmin, d));
+    // limited to the 4-bit range while still a double: floor(x) itself may exceed any integer type
+    double d = fl + (v < frac ? 1.0 : 0.0);
+    return (int)std::min(7.0, std::max((double)dmin, d));
 }
 
 // The default contract: v = (word >> 8) / 2^24.
@@ -167,8 +168,8 @@ Sample sample_noise(uint64_t seed, uint64_t J, float sig, int tier, double tau, 
         double x = (double)sig * R * (odd ? std::sin(th) : std::cos(th));
         double fl = std::floor(x);
         double frac = x - fl;
-        int d = (int)fl + (v < frac ? 1 : 0);
-        out.delta = std::min(7, std::max(dmin, d));
+        double d = fl + (v < frac ? 1.0 : 0.0);
+        out.delta = (int)std::min(7.0, std::max((double)dmin, d));
         out.x = x;
         out.near = (frac < tau) || (frac > 1.0 - tau) || (std::fabs(frac - v) < tau);
     }
@@ -231,11 +232,16 @@ struct Tensor { int32_t bits, qmin, qmax, group_size; int64_t rows, cols; uint64
 // read as binary16, all arithmetic as before; the caller rounds the returned e back to binary16.
 struct HParams { float sigma, lr, gamma; int32_t n_pop, sigma_unit, boundary_mode, antithetic, residual_f16, noise_mode; };
 
+// sigma in grid steps.  With sigma given in weight units the grid-step sigma of a group is
+// sigma / scale_g (fp32 divide), limited to 2^40: beyond that every non-zero sample already
+// saturates the 4-bit range of delta, and the limit keeps sigma_eff * 0 = 0 when the quotient
+// overflows (a zero scale: sigma / 0 = +inf -> 2^40).  Scales are meant to be positive and finite.
 float sigma_eff(const Tensor& t, const HParams& hp, const uint16_t* scales, int64_t j) {
-    if (hp.sigma_unit == 0) return hp.sigma;                    // sigma in grid steps
+    if (hp.sigma_unit == 0) return hp.sigma;
     int64_t row = j / t.cols, col = j % t.cols;
     int64_t g = (t.group_size > 0) ? row * (t.cols / t.group_size) + col / t.group_size : row;
-    return hp.sigma / half_to_float(scales[g]);                 // sigma in weight units
+    float q = hp.sigma / half_to_float(scales[g]);
+    return q < 0x1p40f ? q : 0x1p40f;
 }
 
 // Eq. 4 (GATE) or saturation (CLAMP): the step actually applied to code w.
@@ -268,7 +274,9 @@ template <class F> void parallel_for(int64_t n, int nthreads, F body) {
     for (auto& x : th) x.join();
 }
 
-struct ElemResult { int w_new; double e_new; double band; int gate_final; int gate_replay; int attempted; };
+// blocked: bit k set when the boundary rule blocked or shortened the rounded step of generation k
+// (generations 64 and up are not recorded).
+struct ElemResult { int w_new; double e_new; double band; int gate_final; int gate_replay; int attempted; uint64_t blocked; };
 
 // Algorithm 2 for one element (Algorithm 1 when gens == 1 and e0 is the stored
 // residual).  gens generations, oldest first; the last one is the real update
@@ -281,7 +289,7 @@ ElemResult element_update(const Tensor& t, const HParams& hp, const uint16_t* sc
     const int N = hp.n_pop;
     const double c = (double)hp.lr / ((double)N * (double)hp.sigma);
     const double gamma = (double)hp.gamma;
-    ElemResult r{w, e0, 0.5, 0, 0, 0};
+    ElemResult r{w, e0, 0.5, 0, 0, 0, 0ull};
     double e = e0;
     for (int k = 0; k < gens; ++k) {
         double S = 0.0;
@@ -304,6 +312,7 @@ ElemResult element_update(const Tensor& t, const HParams& hp, const uint16_t* sc
         r.band = std::min(r.band, dist);
         long long applied = applied_step(w, (long long)step, t.qmin, t.qmax, hp.boundary_mode);
         bool blocked = applied != (long long)step;
+        if (blocked && k < 64) r.blocked |= 1ull << k;
         e = u - (double)applied;                                               // Eq. 8 with the gated step
         bool last = (k == gens - 1) && !replay_only;
         if (last) {
@@ -360,6 +369,20 @@ void qo_delta(uint64_t seed, const uint64_t* J, int64_t n, float sigma_eff_v, in
     }
 }
 
+// delta of the even and the odd element of pairs given their four Philox output words (default
+// noise mode: word 0 -> radius, word 1 -> angle, words 2 / 3 -> the two Bernoulli uniforms), tier 1.
+void qo_pair_deltas(const uint32_t* r0, const uint32_t* r1, const uint32_t* r2, const uint32_t* r3, int64_t n,
+                    float sigma_eff_v, int dmin, int32_t* delta_even, int32_t* delta_odd) {
+    for (int64_t i = 0; i < n; ++i) {
+        float R = bm24_radius(r0[i]);
+        float cs, sn;
+        bm24_cossin(r1[i], &cs, &sn);
+        float rho = sigma_eff_v * R;
+        delta_even[i] = stochastic_round_f32(rho * cs, r2[i], dmin);
+        delta_odd[i] = stochastic_round_f32(rho * sn, r3[i], dmin);
+    }
+}
+
 void qo_unpack(int bits, const uint8_t* packed, int64_t n, int32_t* codes) {
     for (int64_t j = 0; j < n; ++j) codes[j] = load_code(packed, bits, j);
 }
@@ -396,12 +419,12 @@ int qo_perturb(const Tensor* t, const uint8_t* w, const uint16_t* scales, uint64
 // Outputs (each nullable except w_new): new code, residual after the step,
 // smallest distance of any generation's u to a rounding boundary, whether the
 // final step was blocked, number of blocked replay steps, whether the final
-// rounded step was non-zero.
+// rounded step was non-zero, and the per-generation record of blocked steps (bit k).
 int qo_update(const Tensor* t, const uint8_t* w, const uint16_t* scales, const uint64_t* seeds,
               const float* fitness, int K, const void* residual_in, const HParams* hp, int tier,
               const int64_t* idx, int64_t n, int nthreads,
               int32_t* w_new, double* e_new, double* band, uint8_t* gate_final, int32_t* gate_replay,
-              uint8_t* attempted) {
+              uint8_t* attempted, uint64_t* blocked) {
     int rc = check(*t, *hp);
     if (rc) return rc;
     if (K < 0) return -5;
@@ -421,6 +444,7 @@ int qo_update(const Tensor* t, const uint8_t* w, const uint16_t* scales, const u
             if (gate_final) gate_final[i] = (uint8_t)r.gate_final;
             if (gate_replay) gate_replay[i] = r.gate_replay;
             if (attempted) attempted[i] = (uint8_t)r.attempted;
+            if (blocked) blocked[i] = r.blocked;
         }
     });
     return 0;
@@ -430,7 +454,7 @@ int qo_update(const Tensor* t, const uint8_t* w, const uint16_t* scales, const u
 int qo_replay_residual(const Tensor* t, const uint8_t* w, const uint16_t* scales, const uint64_t* seeds,
                        const float* fitness, int K, const HParams* hp, int tier,
                        const int64_t* idx, int64_t n, int nthreads,
-                       double* e_out, double* band, int32_t* gate_replay) {
+                       double* e_out, double* band, int32_t* gate_replay, uint64_t* blocked) {
     int rc = check(*t, *hp);
     if (rc) return rc;
     if (K < 0) return -5;
@@ -442,6 +466,7 @@ int qo_replay_residual(const Tensor* t, const uint8_t* w, const uint16_t* scales
             e_out[i] = r.e_new;
             if (band) band[i] = r.band;
             if (gate_replay) gate_replay[i] = r.gate_replay;
+            if (blocked) blocked[i] = r.blocked;
         }
     });
     return 0;

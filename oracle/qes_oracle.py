@@ -161,6 +161,15 @@ def delta(seed: int, J, sigma_eff: float, tier: int = TIER_SPEC, tau: float = 0.
     return d, x, near
 
 
+def pair_deltas(r0, r1, r2, r3, sigma_eff: float, dmin: int = -8):
+    """delta of the even and odd element of pairs from their four Philox words (default noise mode, tier 1)."""
+    r0, r1, r2, r3 = (_arr(r, np.uint32) for r in (r0, r1, r2, r3))
+    n = r0.size
+    de = np.empty(n, np.int32); do = np.empty(n, np.int32)
+    lib().qo_pair_deltas(_p(r0), _p(r1), _p(r2), _p(r3), C.c_int64(n), C.c_float(sigma_eff), C.c_int(dmin), _p(de), _p(do))
+    return de, do
+
+
 def unpack(bits: int, packed, n: int) -> np.ndarray:
     packed = _arr(packed, np.uint8)
     out = np.empty(n, np.int32)
@@ -214,7 +223,8 @@ def update(t: Tensor, w, scales, seeds, fitness, K: int, hp: HParams, residual_i
 
     Returns a dict: w_new int32, e_new float64, band float64 (smallest distance of any
     generation's pre-rounding value to a rounding boundary), gate_final uint8,
-    gate_replay int32, attempted uint8 -- one entry per requested element.
+    gate_replay int32, attempted uint8, blocked uint64 (bit k: the boundary rule blocked or
+    shortened generation k's rounded step) -- one entry per requested element.
     """
     w = _arr(w, np.uint8); s = _scales(scales); idx, n = _idx(idx, t)
     seeds = _arr(seeds, np.uint64).reshape(-1); fitness = _arr(fitness, np.float32).reshape(-1)
@@ -229,13 +239,13 @@ def update(t: Tensor, w, scales, seeds, fitness, K: int, hp: HParams, residual_i
         res = _arr(residual_in, np.float32)
     out = dict(w_new=np.empty(n, np.int32), e_new=np.empty(n, np.float64), band=np.empty(n, np.float64),
                gate_final=np.empty(n, np.uint8), gate_replay=np.empty(n, np.int32),
-               attempted=np.empty(n, np.uint8))
+               attempted=np.empty(n, np.uint8), blocked=np.empty(n, np.uint64))
     tc, hc = t.c(), hp.c()
     rc = lib().qo_update(C.byref(tc), _p(w), _p(s), _p(seeds), _p(fitness), C.c_int(K), _p(res),
                          C.byref(hc), C.c_int(tier), _p(idx), C.c_int64(n),
                          C.c_int(nthreads or default_threads()),
                          _p(out["w_new"]), _p(out["e_new"]), _p(out["band"]), _p(out["gate_final"]),
-                         _p(out["gate_replay"]), _p(out["attempted"]))
+                         _p(out["gate_replay"]), _p(out["attempted"]), _p(out["blocked"]))
     if rc:
         raise ValueError(f"oracle rejected arguments ({rc})")
     return out
@@ -246,12 +256,13 @@ def replay_residual(t: Tensor, w, scales, seeds, fitness, K: int, hp: HParams,
     w = _arr(w, np.uint8); s = _scales(scales); idx, n = _idx(idx, t)
     seeds = _arr(seeds, np.uint64).reshape(-1); fitness = _arr(fitness, np.float32).reshape(-1)
     assert fitness.size == K * hp.n_pop and seeds.size == fitness.size // (2 if hp.antithetic else 1)
-    out = dict(e=np.empty(n, np.float64), band=np.empty(n, np.float64), gate_replay=np.empty(n, np.int32))
+    out = dict(e=np.empty(n, np.float64), band=np.empty(n, np.float64), gate_replay=np.empty(n, np.int32),
+               blocked=np.empty(n, np.uint64))
     tc, hc = t.c(), hp.c()
     rc = lib().qo_replay_residual(C.byref(tc), _p(w), _p(s), _p(seeds), _p(fitness), C.c_int(K),
                                   C.byref(hc), C.c_int(tier), _p(idx), C.c_int64(n),
                                   C.c_int(nthreads or default_threads()),
-                                  _p(out["e"]), _p(out["band"]), _p(out["gate_replay"]))
+                                  _p(out["e"]), _p(out["band"]), _p(out["gate_replay"]), _p(out["blocked"]))
     if rc:
         raise ValueError(f"oracle rejected arguments ({rc})")
     return out

@@ -139,3 +139,26 @@ def test_expected_delta_equals_sigma_eps(qo):
     assert abs(resid.mean()) < 4 * 0.5 / np.sqrt(n)
     assert np.all((resid > -1.0) & (resid <= 1.0))
     assert abs(np.corrcoef(resid, x)[0, 1]) < 4 / np.sqrt(n)
+
+
+def test_pair_deltas_is_delta_on_the_words_philox_produces(qo):
+    """pair_deltas (Box-Muller + Eq. 3 on given words) composed with Philox is delta(seed, J); and on its own
+    it follows Eq. 3 when the uniform word is moved across the exact threshold."""
+    seed = 0x0BADC0DE_CAFEF00D
+    pairs = np.array([0, 1, 77, (1 << 32) + 5, (1 << 39) + 1], dtype=np.uint64)
+    words = np.stack([qo.philox4x32_10([int(p) & 0xffffffff, int(p) >> 32, 0, 0], [seed & 0xffffffff, seed >> 32])
+                      for p in pairs])
+    for sig, dmin in ((0.5, -8), (1.7, -8), (3.0, -7)):
+        de, do = qo.pair_deltas(words[:, 0], words[:, 1], words[:, 2], words[:, 3], sig, dmin)
+        J = np.stack([2 * pairs, 2 * pairs + 1], axis=1).reshape(-1)
+        want = qo.delta(seed, J, sig, dmin=dmin)[0].reshape(-1, 2)
+        assert np.array_equal(de, want[:, 0]) and np.array_equal(do, want[:, 1])
+    # threshold: x = sigma * R * cos with the uniform just below / at the exact fraction
+    r0, r1 = words[:1, 0], words[:1, 1]
+    R, c, _ = qo.bm24(r0, r1)
+    x = Fraction(float(np.float32(np.float32(0.5) * R[0]) * c[0]))
+    fl = x.numerator // x.denominator
+    k = -((-(x - fl) * (1 << 24)).__floor__())          # ceil(frac * 2^24): uniforms 0 .. k-1 give b = 1
+    below = np.array([(k - 1) << 8], np.uint32); at = np.array([k << 8], np.uint32)
+    assert qo.pair_deltas(r0, r1, below, below, 0.5)[0][0] == fl + 1
+    assert qo.pair_deltas(r0, r1, at, at, 0.5)[0][0] == fl
