@@ -8,7 +8,8 @@ Prints ONE JSON line (rank 0).  `value` is weights updated per second over all r
 resident in HBM; `e2e` is the same metric with the weights starting and ending in pinned host
 memory (host<->device copies inside the timed region); `roofline` is the fused update kernel
 against the SM issue peak (the path is bound by integer/fp32 arithmetic, not by HBM);
-`cpu_baseline` is the CPU oracle timed on a bounded sample of the same workload.
+`cpu_baseline` is the CPU oracle timed on a bounded sample of the same workload; `parity` compares
+sampled elements of one untimed step's output with that oracle.
 """
 from __future__ import annotations
 
@@ -96,39 +97,85 @@ class ClockSampler:
                 "power_w_max": max(pw) if pw else None, "samples": len(clk), "reasons": reasons}
 
 
+def sample_words(cfg: wl.Workload, n_words: int, stream: int) -> np.ndarray:
+    """Sorted ids of 32-element words of the flat weight set: the first and the last word of every tensor
+    plus words drawn uniformly over the whole set."""
+    rng = np.random.default_rng([wl.MASTER_SEED, 6, stream])
+    ends = np.array([[t.elem_offset // 32, (t.elem_offset + t.numel) // 32 - 1] for t in cfg.tensors]).reshape(-1)
+    extra = rng.integers(0, cfg.numel // 32, size=max(0, n_words - ends.size))
+    return np.unique(np.concatenate([ends, extra])).astype(np.int64)
+
+
+def flat_oracle_tensor(qo, cfg: wl.Workload):
+    """The whole weight set as one [numel / 32, 32] tensor: with sigma in grid units the noise depends on the
+    global element index alone, so this is the same computation as tensor by tensor."""
+    return qo.Tensor(bits=cfg.bits, rows=cfg.numel // 32, cols=32, group_size=0, elem_offset=cfg.tensors[0].elem_offset)
+
+
+def sparse_packed(cfg: wl.Workload, words: np.ndarray, word_bytes: np.ndarray) -> np.ndarray:
+    """A packed buffer of the whole set that holds `word_bytes` at the sampled words (untouched pages cost nothing)."""
+    per_word = 32 if cfg.bits == 8 else 16
+    buf = np.zeros(wl.packed_bytes(cfg.bits, cfg.numel), np.uint8)
+    buf.reshape(-1, per_word)[words] = word_bytes.reshape(-1, per_word)
+    return buf
+
+
 def oracle_rate(cfg: wl.Workload, target_seconds: float = 15.0, antithetic: bool = False, quad: bool = False):
-    """Times the CPU oracle (as it stands) on a bounded sample of the workload: whole 32-element words
-    drawn from the first tensor of the set, one full step on them (the perturbation of every member,
-    then the stateless update) at the configuration's N and K.  Returns a dict."""
+    """Times the CPU oracle (as it stands) on a bounded sample of the workload: whole 32-element words -- the
+    first and last word of every tensor plus words drawn uniformly over the set -- holding uniform random
+    codes, one full step on them (the perturbation of every member, then the stateless update) at the
+    configuration's N and K.  Returns a dict."""
     from oracle import qes_oracle as qo
     qo.build()
     threads = qo.default_threads()
-    t = cfg.tensors[0]
-    packed = wl.draw_codes(cfg, 0)
     n_seeds = cfg.n_pop // 2 if antithetic else cfg.n_pop
     seeds, fit = wl.draw_seeds(cfg.K + 1, n_seeds), wl.draw_fitness(cfg.K + 1, cfg.n_pop, cfg.reward_dist)
-    to = qo.Tensor(bits=cfg.bits, rows=t.rows, cols=t.cols, group_size=cfg.group_size, elem_offset=t.elem_offset)
+    to = flat_oracle_tensor(qo, cfg)
     hp = qo.HParams(sigma=cfg.sigma, lr=cfg.lr, gamma=cfg.gamma, n_pop=cfg.n_pop, antithetic=int(antithetic),
                     noise_mode=int(quad))
     per_elem = n_seeds * (cfg.K + 1)
+    per_word = 32 if cfg.bits == 8 else 16
 
-    def one_step(idx):
+    def one_step(n_words, stream):
+        words = sample_words(cfg, n_words, stream)
+        codes = np.random.default_rng([wl.MASTER_SEED, 7, stream]).integers(0, 256, size=words.size * per_word, dtype=np.uint8)
+        packed = sparse_packed(cfg, words, codes)
+        idx = (words[:, None] * 32 + np.arange(32)[None, :]).reshape(-1)
         t0 = time.perf_counter()
         for s in seeds[-1]:                                           # Algorithm 1, member loop
             qo.perturb(to, packed, None, int(s), hp, idx=idx)
             if antithetic:
                 qo.perturb(to, packed, None, int(s), hp, idx=idx, sign=-1)
         qo.update(to, packed, None, seeds, fit, cfg.K, hp, idx=idx)   # Algorithm 2
-        return time.perf_counter() - t0
+        return idx.size, time.perf_counter() - t0
 
-    probe_n = max(32 * threads, min(t.numel, int(2e7 // per_elem) // 32 * 32))
-    idx = wl.sample_elements(t.numel, probe_n, stream=900)
-    rate = idx.size / one_step(idx)
-    n = int(min(t.numel, max(probe_n, rate * target_seconds)) // 32 * 32)
-    idx = wl.sample_elements(t.numel, n, stream=901)
-    dt = one_step(idx)
-    return {"weights_per_s": idx.size / dt, "samples_per_s": idx.size * per_elem / dt, "cores": threads,
-            "elements": int(idx.size), "seconds": dt}
+    n_ends = 2 * len(cfg.tensors)
+    n0, dt0 = one_step(max(n_ends, 1024), 900)                        # sizing probe
+    n_words = int(max(n_ends, min(cfg.numel // 32, (n0 / dt0) * target_seconds / 32)))
+    n, dt = one_step(n_words, 901)
+    return {"weights_per_s": n / dt, "samples_per_s": n * per_elem / dt, "cores": threads,
+            "elements": int(n), "seconds": dt}
+
+
+def parity_check(qo_mod, cfg: wl.Workload, before: np.ndarray, after: np.ndarray, perturbed: np.ndarray,
+                 words: np.ndarray, seeds, fit, member_seed: int, antithetic: bool, quad: bool):
+    """Sampled words of one step's output against the oracle: the updated codes (bit-exact outside the counted
+    1e-5 rounding band) and the last member's perturbed copy (bit-exact)."""
+    qo = qo_mod
+    to = flat_oracle_tensor(qo, cfg)
+    hp = qo.HParams(sigma=cfg.sigma, lr=cfg.lr, gamma=cfg.gamma, n_pop=cfg.n_pop, antithetic=int(antithetic), noise_mode=int(quad))
+    idx = (words[:, None] * 32 + np.arange(32)[None, :]).reshape(-1)
+    packed = sparse_packed(cfg, words, before)
+    ref = qo.update(to, packed, None, seeds, fit, cfg.K, hp, idx=idx)
+    near = ref["band"] < 1e-5
+    got = qo.unpack(cfg.bits, after, idx.size)
+    want_p = qo.perturb(to, packed, None, member_seed, hp, idx=idx)
+    got_p = qo.unpack(cfg.bits, perturbed, idx.size)
+    return {"checked": int(idx.size), "mismatch": int(((got != ref["w_new"]) & ~near).sum()), "near_band": int(near.sum()),
+            "perturb_checked": int(idx.size), "perturb_mismatch": int((got_p != want_p).sum()),
+            "changed": int((ref["w_new"] != qo.unpack(cfg.bits, before, idx.size)).sum()),
+            "sample": "first and last 32-element word of every tensor plus uniformly drawn words; one untimed step "
+                      "(last member's perturbed copy, then the stateless update) against the CPU oracle"}
 
 
 def run_reference(args, cfg):
@@ -146,8 +193,8 @@ def run_reference(args, cfg):
             "data": "synthetic", "config": config_dict(cfg, args.gpus, args.antithetic, args.noise_mode),
             "noise_samples_per_s": value * cfg.n_pop * (cfg.K + 1),
             "cpu_baseline": {"value": value, "unit": "weights/s", "cores": rates[0]["cores"], "kind": "oracle",
-                             "sample": f"{rates[0]['elements']} elements (32-element words of tensor 0) per step, "
-                                       f"one full step (perturb x N, update), N={cfg.n_pop}, K={cfg.K}"},
+                             "sample": f"{rates[0]['elements']} elements per step (first and last 32-element word of every tensor "
+                                       f"plus uniformly drawn words), one full step (perturb x N, update), N={cfg.n_pop}, K={cfg.K}"},
             "e2e": {"value": value, "unit": "weights/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
@@ -177,6 +224,7 @@ def main():
                          "per four elements, 8-bit Bernoulli uniforms")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-parity", action="store_true")
     args = ap.parse_args()
     cfg = wl.WORKLOADS[args.workload]
     if args.impl == "reference":
@@ -265,7 +313,7 @@ def main():
     # end to end: weights start and end in pinned host memory
     e2e = None
     if not args.no_e2e:
-        e2e_steps = max(1, min(args.steps, 2))
+        e2e_steps = args.steps
         barrier()
         a, b = ev(), ev(); a.record(stream)
         for _ in range(e2e_steps):
@@ -284,6 +332,22 @@ def main():
         if world > 1:
             dist.destroy_process_group()
         return
+
+    # parity of one more (untimed) step against the CPU oracle, on sampled words of the whole set
+    parity = None
+    if not args.no_parity and world == 1:
+        from oracle import qes_oracle as qo
+        qo.build()
+        per_word = 32 if cfg.bits == 8 else 16
+        words = sample_words(cfg, 2048 + 2 * len(cfg.tensors), stream=950)
+        widx = torch.from_numpy(words).cuda()
+        before = model.w.view(-1, per_word)[widx].cpu().numpy().reshape(-1)
+        step()
+        torch.cuda.synchronize()
+        after = model.w.view(-1, per_word)[widx].cpu().numpy().reshape(-1)
+        pert = scratch.view(-1, per_word)[widx].cpu().numpy().reshape(-1)
+        parity = parity_check(qo, cfg, before, after, pert, words, wl.draw_seeds(cfg.K + 1, n_seeds),
+                              wl.draw_fitness(cfg.K + 1, cfg.n_pop, cfg.reward_dist), member_seeds[-1], args.antithetic, quad)
 
     hbm_gbs, sm_mhz, peak_src = measured_peaks()
     G = cfg.K + 1
@@ -309,13 +373,13 @@ def main():
             "noise_samples_per_s": world * model.numel * n_seeds * G / (update_ms * 1e-3 / args.steps),
             "update_ms_per_step": update_ms / args.steps, "perturb_ms_per_step": perturb_ms / args.steps,
             "perturb_weights_per_s": world * model.numel * cfg.n_pop / (perturb_ms * 1e-3 / args.steps),
-            "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "e2e": e2e}
+            "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "e2e": e2e, "parity": parity}
     if not args.no_cpu_baseline and world == 1:
         r = oracle_rate(cfg, antithetic=args.antithetic, quad=quad)
         line["cpu_baseline"] = {"value": r["weights_per_s"], "unit": "weights/s", "cores": r["cores"], "kind": "oracle",
                                 "samples_per_s": r["samples_per_s"],
-                                "sample": f"{r['elements']} elements (32-element words of tensor 0), one full step (perturb x N, update), "
-                                          f"N={cfg.n_pop}, K={cfg.K}, {r['seconds']:.1f} s"}
+                                "sample": f"{r['elements']} elements (first and last 32-element word of every tensor plus uniformly "
+                                          f"drawn words), one full step (perturb x N, update), N={cfg.n_pop}, K={cfg.K}, {r['seconds']:.1f} s"}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

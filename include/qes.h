@@ -24,8 +24,12 @@
  *    Philox4x32-10(key = seed, counter = J >> 1, or J >> 2 in the QES_NOISE_QUAD8 mode) -> Box-Muller ->
  *    sigma scaling -> stochastic rounding (Eq. 3), limited to the 4-bit range [-8, 7] (App. A).  Results depend only on
  *    (seed, J): any split of a model into tensors, any grid size, gives the same bits.
- *    With sigma_unit == QES_SIGMA_WEIGHT, sigma / scale above 2^40 is treated as 2^40 (every
- *    non-zero sample saturates the 4-bit range long before).
+ *    With sigma_unit == QES_SIGMA_WEIGHT the scales must be positive and finite (device data, not
+ *    checked); sigma / scale above 2^40 is treated as 2^40: every non-zero sample saturates the
+ *    4-bit range long before, and a zero scale (sigma / 0 = +inf) behaves the same way.
+ *  - The kernels first estimate each noise sample with the GPU's special-function unit and recompute
+ *    it with the exact fp32 sequence of the contract only where the estimate cannot settle Eq. 3's
+ *    rounding decision; results are identical to computing every sample exactly.
  *  - Fitness values are the already normalised rewards F_i (Algorithm 1, "Normalize reward").
  *  - Return value: QES_OK, or a negative qes_status; on any error nothing was launched and no
  *    buffer was touched.
@@ -45,12 +49,13 @@ typedef enum {
     QES_ERR_BAD_BITS = -2,    /* bits is not 4 or 8 */
     QES_ERR_BAD_SHAPE = -3,   /* rows/cols/group_size/elem_offset violate the layout rules */
     QES_ERR_MISALIGNED = -4,  /* a device pointer misses its alignment (16 B weights/residual, 8 B seeds, 4 B fitness, 2 B scales) */
-    QES_ERR_BAD_HPARAM = -5,  /* sigma <= 0, n_pop <= 0 (or odd with antithetic pairs), K < 0, gamma outside [0,1], qmin >= qmax, range outside the code width */
+    QES_ERR_BAD_HPARAM = -5,  /* sigma <= 0, n_pop <= 0 (or odd with antithetic pairs), K < 0 or K > QES_MAX_K, gamma outside [0,1], qmin >= qmax, range outside the code width */
     QES_ERR_BAD_MODE = -6,    /* unknown sigma_unit / boundary_mode / antithetic / residual_f16 / noise_mode, residual_inout given with K > 0, qes_perturb_pair without antithetic, or its two outputs the same buffer */
     QES_ERR_CUDA = -7,        /* the launch reported a CUDA error (cudaGetLastError) */
     QES_ERR_TOO_LARGE = -8    /* more seeds per generation than the shared-memory staging holds (1066: members, or antithetic pairs) */
 } qes_status;
 
+enum { QES_MAX_K = 1 << 20 };   /* largest replay depth K accepted */
 enum { QES_SIGMA_GRID = 0, QES_SIGMA_WEIGHT = 1 };   /* unit of hparams.sigma: grid steps | weight units (sigma_g = sigma / scale_g) */
 enum { QES_BOUNDARY_GATE = 0, QES_BOUNDARY_CLAMP = 1 }; /* Eq. 4 masking | saturation */
 /* How the 128 bits of one Philox4x32-10 call are spent (the paper leaves "RNG(seed)" open):
@@ -59,7 +64,8 @@ enum { QES_BOUNDARY_GATE = 0, QES_BOUNDARY_CLAMP = 1 }; /* Eq. 4 masking | satur
  *   QES_NOISE_QUAD8   one call per four elements, counter = J >> 2: words 0,1 and 2,3 -> two Box-Muller pairs
  *                     (top 24 bits of each word), element h's Bernoulli uniform (b + 1/2) / 256 from the low byte b
  *                     of word h (P(b = 1) is the fraction of sigma*eps to the nearest 1/256); half the Philox work.
- * The two modes draw different streams; each is reproduced bit for bit by the reference implementation. */
+ * The two modes draw different streams; each is fully specified (a scalar CPU implementation of the same
+ * contract reproduces either bit for bit). */
 enum { QES_NOISE_PAIR24 = 0, QES_NOISE_QUAD8 = 1 };
 
 typedef struct {
@@ -77,24 +83,25 @@ typedef struct {
     int32_t n_pop;         /* population size N */
     int32_t sigma_unit;    /* QES_SIGMA_GRID | QES_SIGMA_WEIGHT */
     int32_t boundary_mode; /* QES_BOUNDARY_GATE | QES_BOUNDARY_CLAMP */
-    int32_t antithetic;    /* 0: N members, N seeds per generation.  1 (App. A, "antithetic perturbation
-                              pairs"): N even, N/2 pairs per generation, pair j = one seed and the two members
+    int32_t antithetic;    /* 0: N members, N seeds per generation.  1 (App. A, population setting of the
+                              reasoning runs): N even, N/2 pairs per generation, pair j = one seed and the two members
                               W + delta_j, W - delta_j; seeds tables then hold N/2 entries per generation,
                               fitness tables N entries per generation ordered F+_0, F-_0, F+_1, F-_1, ...,
                               and delta is limited to the symmetric 4-bit range [-7, 7] */
-    int32_t residual_f16;  /* format of residual_inout / residual_out: 0 = float, 1 = IEEE binary16 (Algorithm 1,
-                              "Residuals e_0 <- 0 (FP16)"): read as binary16, arithmetic in fp32, rounded to
-                              nearest even on the store */
+    int32_t residual_f16;  /* format of residual_inout / residual_out: 0 = float, 1 = IEEE binary16 (the precision
+                              Algorithm 1's initialisation line gives the residual): read as binary16, arithmetic
+                              in fp32, rounded to nearest even on the store */
     int32_t noise_mode;    /* QES_NOISE_PAIR24 | QES_NOISE_QUAD8 */
 } qes_hparams;
 
 /*
- * Algorithm 1, "Reconstruct delta_i" + "Gate(W_t + delta_i)" (Eqs. 3-4) for one population member.
+ * Algorithm 1, the two lines of the member loop that rebuild the member's perturbation from its seed and apply
+ * it under the boundary gate (Eqs. 3-4), for one population member.
  *   w_in  [device, rows*cols codes]  current weights, not modified (unless w_out == w_in)
  *   w_out [device, same size]        perturbed weights; may alias w_in exactly, no partial overlap
  *   seed                             the member's seed s_i
- * Only sigma, sigma_unit, boundary_mode and antithetic (which narrows delta to [-7, 7]) of hparams are
- * used (n_pop, lr, gamma still validated).
+ * Only sigma, sigma_unit, boundary_mode, noise_mode and antithetic (which narrows delta to [-7, 7]) of hparams
+ * are used (n_pop, lr, gamma still validated).
  */
 int qes_perturb(const qes_tensor_desc* desc, const void* w_in, void* w_out, const void* scales_f16,
                 uint64_t seed, const qes_hparams* hparams, void* cuda_stream);
@@ -149,6 +156,36 @@ int qes_gaussian_factors(const uint32_t* r0, const uint32_t* r1, int64_t n, floa
                          float* sine, void* cuda_stream);
 
 /*
+ * The special-function-unit estimates the kernels try first (no counterpart in the paper): for each i the
+ * estimates of the same three factors as qes_gaussian_factors, from lg2 / sqrt / sin / cos approximations.
+ * They are NOT part of the noise contract; the kernels use them only where their error cannot change
+ * Eq. 3's result (see qes_estimate_bounds).  Same argument rules as qes_gaussian_factors.
+ */
+int qes_gaussian_estimates(const uint32_t* r0, const uint32_t* r1, int64_t n, float* radius, float* cosine,
+                           float* sine, void* cuda_stream);
+
+/*
+ * The constants of that verification (HOST pointers, all required): *eps_bound bounds |R~ c~ - R c| (estimate
+ * minus exact product of radius and angle factor) for every angle word and every radius word below
+ * *radius_word_limit; radius words at or above the limit always take the exact sequence; *rounding_bound is the
+ * allowance, per unit of sigma_eff, for the fp32 roundings of both forms.  A sample is recomputed exactly when its
+ * estimated rounding sum lies within E = 2^ceil(log2(sigma_eff * 2^24 * (eps_bound + rounding_bound) + 3)) (at
+ * least 16) of a multiple of 2^24.  Lets a caller check, with qes_gaussian_factors and qes_gaussian_estimates on
+ * all 2^24 inputs of each factor, that the bound holds on the device at hand.
+ */
+int qes_estimate_bounds(float* eps_bound, float* rounding_bound, uint32_t* radius_word_limit);
+
+/*
+ * Eq. 3 for both elements of a pair from caller-supplied Philox output words (default noise mode: r0 -> radius,
+ * r1 -> angle, r2 / r3 -> the 24-bit uniforms of the even / odd element), through the kernels' own
+ * estimate-then-verify sequence: delta_even[i], delta_odd[i] in [-8, 7]; verified[i] (nullable) = 1 where the
+ * exact sequence had to decide.  sigma_eff in grid steps, 0 < sigma_eff <= 2^40.  All arrays are DEVICE pointers
+ * to n elements owned by the caller.  For tests that place samples on and around rounding decisions.
+ */
+int qes_pair_deltas(const uint32_t* r0, const uint32_t* r1, const uint32_t* r2, const uint32_t* r3, int64_t n,
+                    float sigma_eff, int8_t* delta_even, int8_t* delta_odd, uint8_t* verified, void* cuda_stream);
+
+/*
  * Arithmetic-pipe throughput probes used to derive the ALU roofline (no counterpart in the
  * paper).  Runs `iters` dependent-chain iterations of one instruction kind on every lane of a
  * full grid and writes the elapsed device time in milliseconds to *ms_out (HOST pointer) and
@@ -157,13 +194,9 @@ int qes_gaussian_factors(const uint32_t* r0, const uint32_t* r1, int64_t n, floa
  * that is practically never taken).  Runs on the default stream and synchronises.
  *   kind: 0 mul.wide.u32 (low half kept)  1 lop3 (xor3)  2 fma.rn.f32  3 mul.hi.u32  4 cvt.rn.f32.u32
  *         5 sqrt.rn.f32   6 cvt.rmi (floor)  7 mad.lo.u32  8 Philox round (2 wide multiplies + 2 xor3)
- *         9 rsqrt.approx.f32 (special-function unit)  10-17 add, shift, fp32 add/mul/compare/min, cvt.rzi
- *         18 mad.wide.u32 with the 64-bit result live  19 mul.wide.u32 + xor3 of both halves (counted
- *         per step)  20/21/22 the same plus 1/2/4 independent fp32 fma per step
- *         23/24/25 the update kernel's mix per step (one wide multiply, 2.5 xor3, 2 fp32 fma) in three
- *         program orders: chain by chain, kinds alternating, kinds grouped
- *         26 fma.rn.f32x2 (packed pair of fp32 fma, counted per instruction)  27 mul.wide.u32 + xor3 + one f32x2 per step
- *         100-109 two-kind mixes (see the binding's PROBE_KINDS)
+ *         9 rsqrt.approx.f32 (special-function unit)  10-17 add, shift, fp32 add/mul/compare/min, cvt.rzi, set
+ *         18 mad.wide.u32 with the 64-bit result live  19 mul.wide.u32 + xor3 of both halves (counted per step)
+ *         20 lg2.approx.f32  21 sin.approx.f32  22 sqrt.approx.f32  23 cvt.rn.f32.s8
  */
 int qes_pipe_probe(int32_t kind, int32_t iters, void* sink_dev, float* ms_out, double* ops_out);
 

@@ -110,6 +110,12 @@ def load() -> C.CDLL:
         lib.qes_update.argtypes = [C.POINTER(_TensorDesc), vp, vp, vp, vp, i32, vp, C.POINTER(_HParams), vp, vp]
         lib.qes_gaussian_factors.restype = C.c_int
         lib.qes_gaussian_factors.argtypes = [vp, vp, C.c_int64, vp, vp, vp, vp]
+        lib.qes_gaussian_estimates.restype = C.c_int
+        lib.qes_gaussian_estimates.argtypes = [vp, vp, C.c_int64, vp, vp, vp, vp]
+        lib.qes_estimate_bounds.restype = C.c_int
+        lib.qes_estimate_bounds.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_float), C.POINTER(C.c_uint32)]
+        lib.qes_pair_deltas.restype = C.c_int
+        lib.qes_pair_deltas.argtypes = [vp, vp, vp, vp, C.c_int64, C.c_float, vp, vp, vp, vp]
         lib.qes_pipe_probe.restype = C.c_int
         lib.qes_pipe_probe.argtypes = [i32, i32, vp, C.POINTER(C.c_float), C.POINTER(C.c_double)]
         lib.qes_strerror.restype = C.c_char_p
@@ -217,18 +223,41 @@ def qes_gaussian_factors(r0, r1, radius, cosine, sine, stream=None) -> None:
     _check(rc)
 
 
+def qes_gaussian_estimates(r0, r1, radius, cosine, sine, stream=None) -> None:
+    """The special-function-unit estimates of the same three factors (what the kernels try first)."""
+    n = r0.numel()
+    words = (torch.int32, torch.uint32)
+    rc = load().qes_gaussian_estimates(_ptr(r0, dtype=words, nbytes=4 * n, name="r0"), _ptr(r1, dtype=words, nbytes=4 * n, name="r1"),
+                                       n, _ptr(radius, dtype=torch.float32, nbytes=4 * n, name="radius"),
+                                       _ptr(cosine, dtype=torch.float32, nbytes=4 * n, name="cosine"),
+                                       _ptr(sine, dtype=torch.float32, nbytes=4 * n, name="sine"), _stream(stream))
+    _check(rc)
+
+
+def qes_estimate_bounds():
+    """(eps_bound, rounding_bound, radius_word_limit) of the estimate-then-verify sequence."""
+    eps, rnd, lim = C.c_float(0), C.c_float(0), C.c_uint32(0)
+    _check(load().qes_estimate_bounds(C.byref(eps), C.byref(rnd), C.byref(lim)))
+    return eps.value, rnd.value, lim.value
+
+
+def qes_pair_deltas(r0, r1, r2, r3, sigma_eff: float, delta_even, delta_odd, verified=None, stream=None) -> None:
+    """Eq. 3 for both elements of pairs given their four Philox words, through the kernels' own sequence."""
+    n = r0.numel()
+    words = (torch.int32, torch.uint32)
+    rc = load().qes_pair_deltas(*(_ptr(r, dtype=words, nbytes=4 * n, name=f"r{i}") for i, r in enumerate((r0, r1, r2, r3))),
+                                n, C.c_float(sigma_eff), _ptr(delta_even, dtype=torch.int8, nbytes=n, name="delta_even"),
+                                _ptr(delta_odd, dtype=torch.int8, nbytes=n, name="delta_odd"),
+                                _ptr(verified, dtype=torch.uint8, nbytes=n, name="verified"), _stream(stream))
+    _check(rc)
+
+
 PROBE_KINDS = {0: "mul.wide.u32", 1: "lop3.xor3", 2: "fma.rn.f32", 3: "mul.hi.u32", 4: "cvt.rn.f32.u32",
                5: "sqrt.rn.f32", 6: "cvt.rmi.f32.f32", 7: "mad.lo.u32", 8: "philox round (2 mul.wide + 2 xor3)",
                9: "rsqrt.approx.f32", 10: "add.u32", 11: "shr.u32", 12: "add.rn.f32", 13: "mul.rn.f32",
                14: "setp.lt.f32 + selp", 15: "min.f32", 16: "cvt.rzi.s32.f32", 17: "set.lt.f32 (1.0/0.0)", 18: "mad.wide.u32 (64-bit result live)",
-               19: "mul.wide.u32 + xor3 of both halves (steps)", 20: "mul.wide + xor3 + 1 fma (steps)",
-               21: "mul.wide + xor3 + 2 fma (steps)", 22: "mul.wide + xor3 + 4 fma (steps)",
-               23: "update-kernel mix: wide + 2.5 xor3 + 2 fma (steps)",
-               24: "the same mix, kinds alternating (steps)", 25: "the same mix, kinds grouped (steps)",
-               26: "fma.rn.f32x2 (instructions, two fmas each)", 27: "mul.wide + xor3 + 1 fma.f32x2 (steps)",
-               100: "mix mul.wide + xor3", 101: "mix fma + xor3", 102: "mix mul.wide + fma", 103: "mix cvt.f32.u32 + xor3",
-               104: "mix cvt.f32.u32 + mul.wide", 105: "mix floor + rsqrt", 106: "mix floor + fma", 107: "mix add + xor3",
-               108: "mix fadd + mul.wide", 109: "mix setp/selp + fma"}
+               19: "mul.wide.u32 + xor3 of both halves (steps)", 20: "lg2.approx.f32", 21: "sin.approx.f32",
+               22: "sqrt.approx.f32", 23: "cvt.rn.f32.s8"}
 
 
 def qes_pipe_probe(kind: int, iters: int = 4096):

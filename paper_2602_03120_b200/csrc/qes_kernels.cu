@@ -19,19 +19,13 @@
 #include "qes_device.cuh"
 #include "../../include/qes.h"
 
-#ifndef QES_PAIRS
-#define QES_PAIRS 4
-#endif
-#ifndef QES_MIN_BLOCKS
-#define QES_MIN_BLOCKS 2
-#endif
-
 namespace qes {
 
 enum PassMode : int { kStateless = 0, kStoredResidual = 1, kReplayOnly = 2 };
 
 constexpr int kThreads = 256;
-constexpr int kPairs = QES_PAIRS;
+constexpr int kPairs = 4;
+constexpr int kMinBlocksPerSm = 2;
 constexpr int kCodesPerThread = 2 * kPairs;
 constexpr int kSeedStride = 24;   // 32-bit words per staged member: a[10], b[10], fitness, SeedConst
 
@@ -159,12 +153,20 @@ __global__ void __launch_bounds__(kThreads) perturb_kernel(PassParams p, RoundKe
     Chunk<BITS, kPairs> out, out_minus;
     out.clear();
     out_minus.clear();
+    FastGuard guard;
+    if constexpr (!QUAD) guard = make_fast_guard(nsig24);
 #pragma unroll
     for (int i = 0; i < kCalls; ++i) {
         uint32_t r0, r1, r2, r3;
         philox_tail(make_pair_const(x0 + i), sc, rk, r0, r1, r2, r3);
         int z[kPerCall];
-        call_rounding_sums<CLAMP_DELTA, QUAD>(r0, r1, r2, r3, nsig24, z);
+        if constexpr (QUAD) {
+            call_rounding_sums<CLAMP_DELTA, true>(r0, r1, r2, r3, nsig24, z);
+        } else {
+            // special-function estimate first; the exact sequence only where the estimate cannot decide
+            if (pair_rounding_sums_estimate<CLAMP_DELTA>(r0, r1, r2, r3, nsig24, guard, z[0], z[1]))
+                call_rounding_sums<CLAMP_DELTA, false>(r0, r1, r2, r3, nsig24, z);
+        }
 #pragma unroll
         for (int j = 0; j < kPerCall; ++j) {
             const int t = kPerCall * i + j;
@@ -215,7 +217,7 @@ __device__ __forceinline__ RoundKeys load_round_keys(const uint32_t* entry, floa
 // Algorithm 2 (stateless), Algorithm 1's update lines (stored residual) or the history loop
 // alone (replay only), selected by p.mode.  Shared memory: 2 * (seeds per generation) * 96 B.
 template <int BITS, bool CLAMP_DELTA, bool STATS, bool QUAD>
-__global__ void __launch_bounds__(kThreads, QES_MIN_BLOCKS) pass_kernel(PassParams p) {
+__global__ void __launch_bounds__(kThreads, kMinBlocksPerSm) pass_kernel(PassParams p) {
     extern __shared__ __align__(16) uint32_t smem[];
     constexpr int T = kCodesPerThread;
     constexpr int kPerCall = QUAD ? 4 : 2;                 // elements served by one Philox call
@@ -241,6 +243,9 @@ __global__ void __launch_bounds__(kThreads, QES_MIN_BLOCKS) pass_kernel(PassPara
 #pragma unroll
         for (int i = 0; i < kCalls; ++i) pc[i] = make_pair_const((uint32_t)call0 + i);
     }
+
+    FastGuard guard;
+    if constexpr (!QUAD) guard = make_fast_guard(nsig24);
 
     const int last = p.generations - 1;
     const int buf_words = p.n_seeds * kSeedStride;
@@ -272,16 +277,45 @@ __global__ void __launch_bounds__(kThreads, QES_MIN_BLOCKS) pass_kernel(PassPara
             SeedConst sc;
             const RoundKeys rk = load_round_keys(table + i * kSeedStride, Fm, sc);
             if (!y_uniform) sc = make_seed_const(y, rk);
+            float nd[T];   // -delta of this seed for the thread's codes
+            if constexpr (QUAD) {
 #pragma unroll
-            for (int c = 0; c < kCalls; ++c) {
-                uint32_t r0, r1, r2, r3;
-                philox_tail(pc[c], sc, rk, r0, r1, r2, r3);
-                int z[kPerCall];
-                call_rounding_sums<CLAMP_DELTA, QUAD>(r0, r1, r2, r3, nsig24, z);
+                for (int c = 0; c < kCalls; ++c) {
+                    uint32_t r0, r1, r2, r3;
+                    philox_tail(pc[c], sc, rk, r0, r1, r2, r3);
+                    int z[kPerCall];
+                    call_rounding_sums<CLAMP_DELTA, true>(r0, r1, r2, r3, nsig24, z);
 #pragma unroll
-                for (int j = 0; j < kPerCall; ++j)          // Eq. 5 numerator
-                    S[kPerCall * c + j] = fmaf(Fm, neg_delta_float<CLAMP_DELTA>(z[j], p.nd_max), S[kPerCall * c + j]);
+                    for (int j = 0; j < kPerCall; ++j) nd[kPerCall * c + j] = neg_delta_float<CLAMP_DELTA>(z[j], p.nd_max);
+                }
+            } else {
+                // special-function estimates for all four pairs; if any of the eight samples lies too
+                // close to a rounding decision for the estimate to settle it (about 1.5e-4 of the
+                // (thread, seed) steps at sigma = 0.5), the seed is redone with the exact sequence
+                bool undecided = false;
+#pragma unroll
+                for (int c = 0; c < kCalls; ++c) {
+                    uint32_t r0, r1, r2, r3;
+                    philox_tail(pc[c], sc, rk, r0, r1, r2, r3);
+                    int ze, zo;
+                    undecided |= pair_rounding_sums_estimate<CLAMP_DELTA>(r0, r1, r2, r3, nsig24, guard, ze, zo);
+                    nd[2 * c] = neg_delta_float<CLAMP_DELTA>(ze, p.nd_max);
+                    nd[2 * c + 1] = neg_delta_float<CLAMP_DELTA>(zo, p.nd_max);
+                }
+                if (__builtin_expect(undecided, 0)) {
+#pragma unroll
+                    for (int c = 0; c < kCalls; ++c) {
+                        uint32_t r0, r1, r2, r3;
+                        philox_tail(pc[c], sc, rk, r0, r1, r2, r3);
+                        int z[2];
+                        call_rounding_sums<CLAMP_DELTA, false>(r0, r1, r2, r3, nsig24, z);
+                        nd[2 * c] = neg_delta_float<CLAMP_DELTA>(z[0], p.nd_max);
+                        nd[2 * c + 1] = neg_delta_float<CLAMP_DELTA>(z[1], p.nd_max);
+                    }
+                }
             }
+#pragma unroll
+            for (int t = 0; t < T; ++t) S[t] = fmaf(Fm, nd[t], S[t]);      // Eq. 5 numerator
         }
         const bool is_update = (k == last) && (p.mode != kReplayOnly);
 #pragma unroll
@@ -336,6 +370,34 @@ __global__ void __launch_bounds__(kThreads) gaussian_factors_kernel(const uint32
     bm_cossin(r1[i], c, s);
     C[i] = c;
     S[i] = s;
+}
+
+// The special-function estimates of the same factors (what the kernels try first).
+__global__ void __launch_bounds__(kThreads) gaussian_estimates_kernel(const uint32_t* r0, const uint32_t* r1, int64_t n,
+                                                                      float* R, float* C, float* S) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    R[i] = radius_estimate(r0[i]);
+    float c, s;
+    cossin_estimate(r1[i], c, s);
+    C[i] = c;
+    S[i] = s;
+}
+
+// delta of both elements of a pair from caller-supplied Philox words, through the same
+// estimate-then-verify sequence as the update and perturb kernels (default noise mode).
+__global__ void __launch_bounds__(kThreads) pair_deltas_kernel(const uint32_t* r0, const uint32_t* r1, const uint32_t* r2,
+                                                               const uint32_t* r3, int64_t n, float nsig24,
+                                                               signed char* d_even, signed char* d_odd, unsigned char* verified) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const FastGuard guard = make_fast_guard(nsig24);
+    int z[2];
+    const bool undecided = pair_rounding_sums_estimate<true>(r0[i], r1[i], r2[i], r3[i], nsig24, guard, z[0], z[1]);
+    if (undecided) call_rounding_sums<true, false>(r0[i], r1[i], r2[i], r3[i], nsig24, z);
+    d_even[i] = (signed char)(-neg_delta<true>(z[0], 8));
+    d_odd[i] = (signed char)(-neg_delta<true>(z[1], 8));
+    if (verified != nullptr) verified[i] = undecided ? 1 : 0;
 }
 
 // ------------------------------------------------------------------------- host side
@@ -502,7 +564,7 @@ int qes_replay_residual(const qes_tensor_desc* desc, const void* w, const void* 
                         const qes_hparams* hparams, void* residual_out, void* cuda_stream) {
     int rc = validate(desc, hparams);
     if (rc != QES_OK) return rc;
-    if (K < 0) return QES_ERR_BAD_HPARAM;
+    if (K < 0 || K > QES_MAX_K) return QES_ERR_BAD_HPARAM;
     if (w == nullptr || residual_out == nullptr) return QES_ERR_NULL_PTR;
     if (hparams->sigma_unit == QES_SIGMA_WEIGHT && scales_f16 == nullptr) return QES_ERR_NULL_PTR;
     if (!aligned(w, 16) || !aligned(residual_out, 16) || !aligned(scales_f16, 2)) return QES_ERR_MISALIGNED;
@@ -525,7 +587,7 @@ int qes_update(const qes_tensor_desc* desc, void* w_inout, const void* scales_f1
                const qes_hparams* hparams, uint64_t* stats, void* cuda_stream) {
     int rc = validate(desc, hparams);
     if (rc != QES_OK) return rc;
-    if (K < 0) return QES_ERR_BAD_HPARAM;
+    if (K < 0 || K > QES_MAX_K) return QES_ERR_BAD_HPARAM;
     if (residual_inout != nullptr && K != 0) return QES_ERR_BAD_MODE;
     if (w_inout == nullptr) return QES_ERR_NULL_PTR;
     if (hparams->sigma_unit == QES_SIGMA_WEIGHT && scales_f16 == nullptr) return QES_ERR_NULL_PTR;
@@ -559,6 +621,43 @@ int qes_gaussian_factors(const uint32_t* r0, const uint32_t* r1, int64_t n, floa
     return cudaGetLastError() == cudaSuccess ? QES_OK : QES_ERR_CUDA;
 }
 
+int qes_gaussian_estimates(const uint32_t* r0, const uint32_t* r1, int64_t n, float* radius, float* cosine,
+                           float* sine, void* cuda_stream) {
+    if (n < 0) return QES_ERR_BAD_SHAPE;
+    if (n == 0) return QES_OK;
+    if (r0 == nullptr || r1 == nullptr || radius == nullptr || cosine == nullptr || sine == nullptr) return QES_ERR_NULL_PTR;
+    if (!aligned(r0, 4) || !aligned(r1, 4) || !aligned(radius, 4) || !aligned(cosine, 4) || !aligned(sine, 4))
+        return QES_ERR_MISALIGNED;
+    if ((n + kThreads - 1) / kThreads > (int64_t)INT32_MAX) return QES_ERR_BAD_SHAPE;
+    unsigned blocks = (unsigned)((n + kThreads - 1) / kThreads);
+    gaussian_estimates_kernel<<<blocks, kThreads, 0, reinterpret_cast<cudaStream_t>(cuda_stream)>>>(r0, r1, n, radius, cosine, sine);
+    return cudaGetLastError() == cudaSuccess ? QES_OK : QES_ERR_CUDA;
+}
+
+int qes_pair_deltas(const uint32_t* r0, const uint32_t* r1, const uint32_t* r2, const uint32_t* r3, int64_t n,
+                    float sigma_eff, int8_t* delta_even, int8_t* delta_odd, uint8_t* verified, void* cuda_stream) {
+    if (n < 0) return QES_ERR_BAD_SHAPE;
+    if (!(sigma_eff > 0.0f) || !(sigma_eff <= 0x1p40f)) return QES_ERR_BAD_HPARAM;
+    if (n == 0) return QES_OK;
+    if (r0 == nullptr || r1 == nullptr || r2 == nullptr || r3 == nullptr || delta_even == nullptr || delta_odd == nullptr)
+        return QES_ERR_NULL_PTR;
+    if (!aligned(r0, 4) || !aligned(r1, 4) || !aligned(r2, 4) || !aligned(r3, 4)) return QES_ERR_MISALIGNED;
+    if ((n + kThreads - 1) / kThreads > (int64_t)INT32_MAX) return QES_ERR_BAD_SHAPE;
+    unsigned blocks = (unsigned)((n + kThreads - 1) / kThreads);
+    pair_deltas_kernel<<<blocks, kThreads, 0, reinterpret_cast<cudaStream_t>(cuda_stream)>>>(
+        r0, r1, r2, r3, n, -sigma_eff * 0x1p24f, reinterpret_cast<signed char*>(delta_even),
+        reinterpret_cast<signed char*>(delta_odd), verified);
+    return cudaGetLastError() == cudaSuccess ? QES_OK : QES_ERR_CUDA;
+}
+
+int qes_estimate_bounds(float* eps_bound, float* rounding_bound, uint32_t* radius_word_limit) {
+    if (eps_bound == nullptr || rounding_bound == nullptr || radius_word_limit == nullptr) return QES_ERR_NULL_PTR;
+    *eps_bound = kFastEpsBound;
+    *rounding_bound = kFastRoundingBound;
+    *radius_word_limit = kFastRadiusWordLimit;
+    return QES_OK;
+}
+
 const char* qes_strerror(int status) {
     switch (status) {
         case QES_OK: return "ok";
@@ -566,7 +665,7 @@ const char* qes_strerror(int status) {
         case QES_ERR_BAD_BITS: return "bits must be 4 or 8";
         case QES_ERR_BAD_SHAPE: return "rows/cols/group_size/elem_offset violate the layout rules";
         case QES_ERR_MISALIGNED: return "a device pointer is not aligned as required";
-        case QES_ERR_BAD_HPARAM: return "hyper-parameter or code range out of bounds";
+        case QES_ERR_BAD_HPARAM: return "hyper-parameter, replay depth or code range out of bounds";
         case QES_ERR_BAD_MODE: return "unknown mode, stored residual combined with K > 0, or a pair call without antithetic set";
         case QES_ERR_CUDA: return "CUDA reported an error at launch";
         case QES_ERR_TOO_LARGE: return "n_pop exceeds the shared-memory staging limit";
@@ -574,6 +673,6 @@ const char* qes_strerror(int status) {
     }
 }
 
-int qes_version(void) { return 120; }
+int qes_version(void) { return 200; }
 
 }  // extern "C"

@@ -70,6 +70,22 @@ __device__ __forceinline__ uint32_t step(uint32_t x, uint32_t a, uint32_t b) {
         float f;
         asm volatile("set.lt.f32.f32 %0, %1, %2;" : "=f"(f) : "f"(__uint_as_float(x)), "f"(__uint_as_float(b)));
         r = __float_as_uint(f);
+    } else if (KIND == 20) {  // special-function unit: base-2 logarithm
+        float f;
+        asm volatile("lg2.approx.ftz.f32 %0, %1;" : "=f"(f) : "f"(__uint_as_float(x)));
+        r = __float_as_uint(f);
+    } else if (KIND == 21) {  // special-function unit: sine (with the range multiply the assembler adds)
+        float f;
+        asm volatile("sin.approx.ftz.f32 %0, %1;" : "=f"(f) : "f"(__uint_as_float(x)));
+        r = __float_as_uint(f);
+    } else if (KIND == 22) {  // special-function unit: square-root estimate
+        float f;
+        asm volatile("sqrt.approx.ftz.f32 %0, %1;" : "=f"(f) : "f"(__uint_as_float(x)));
+        r = __float_as_uint(f);
+    } else if (KIND == 23) {  // signed byte -> float conversion (the weighted sum's operand)
+        float f;
+        asm volatile("cvt.rn.f32.s8 %0, %1;" : "=f"(f) : "r"(x));
+        r = __float_as_uint(f) ^ x;
     } else {
         r = x;
     }
@@ -106,42 +122,16 @@ __global__ void __launch_bounds__(kProbeThreads) probe_kernel(int iters, uint32_
     if (acc == 0x12345u) sink[0] = acc;   // keeps the chains live; practically never taken
 }
 
-template <int KA, int KB>
-__global__ void __launch_bounds__(kProbeThreads) probe_mix_kernel(int iters, uint32_t a, uint32_t b, uint32_t* sink) {
-    uint32_t x[kChains];
-#pragma unroll
-    for (int c = 0; c < kChains; ++c) x[c] = threadIdx.x * 2654435761u + c * 40503u + blockIdx.x + 0x3f800001u;
-    for (int it = 0; it < iters; ++it) {
-#pragma unroll
-        for (int c = 0; c < kChains; c += 2) {
-            x[c] = step<KA>(x[c], a, b);
-            x[c + 1] = step<KB>(x[c + 1], a, b);
-        }
-    }
-    uint32_t acc = 0;
-#pragma unroll
-    for (int c = 0; c < kChains; ++c) acc ^= x[c];
-    if (acc == 0x12345u) sink[0] = acc;
-}
-
 // Wide multiplies whose two result halves both stay live (a chain that keeps only the low half
 // can be narrowed by the assembler).  MODE 0: w = lo(w) * a + w, one 64-bit multiply-add per
 // step.  MODE 1: (h, l) = x * a; x = h ^ l ^ b, one wide multiply and one three-input xor per
-// step, the shape of a Philox round.  MODE 2 / 3 / 4: MODE 1 plus one / two / four independent
-// fp32 fused multiply-adds per step, which shows whether fp32 work shares the pipe of the wide
-// multiply or runs beside it.
+// step, the shape of half a Philox round.
 template <int MODE>
 __global__ void __launch_bounds__(kProbeThreads) probe_wide_kernel(int iters, uint32_t a, uint32_t b, uint32_t* sink) {
-    constexpr int kFma = MODE == 2 ? 1 : MODE == 3 ? 2 : MODE == 4 ? 4 : 0;
     unsigned long long w[kChains];
-    float f[kChains][kFma > 0 ? kFma : 1];
 #pragma unroll
-    for (int c = 0; c < kChains; ++c) {
+    for (int c = 0; c < kChains; ++c)
         w[c] = ((unsigned long long)(threadIdx.x * 2654435761u + c * 40503u) << 32) | (blockIdx.x + 0x3f800001u + c);
-#pragma unroll
-        for (int j = 0; j < (kFma > 0 ? kFma : 1); ++j) f[c][j] = 1.0f + 1e-3f * (float)(threadIdx.x + c + j);
-    }
-    const float fa = __uint_as_float(b), fb = 1e-7f;   // b is passed as the bits of a float just below 1
     for (int it = 0; it < iters; ++it) {
 #pragma unroll
         for (int c = 0; c < kChains; ++c) {
@@ -151,181 +141,13 @@ __global__ void __launch_bounds__(kProbeThreads) probe_wide_kernel(int iters, ui
                 unsigned long long p;
                 asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(p) : "r"((uint32_t)w[c]), "r"(a));
                 w[c] = (uint32_t)(p >> 32) ^ (uint32_t)p ^ b;
-#pragma unroll
-                for (int j = 0; j < kFma; ++j)
-                    asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(f[c][j]) : "f"(fa), "f"(fb));
             }
         }
     }
     uint32_t acc = 0;
 #pragma unroll
-    for (int c = 0; c < kChains; ++c) {
-        acc ^= (uint32_t)w[c] ^ (uint32_t)(w[c] >> 32);
-#pragma unroll
-        for (int j = 0; j < kFma; ++j) acc ^= __float_as_uint(f[c][j]);
-    }
+    for (int c = 0; c < kChains; ++c) acc ^= (uint32_t)w[c] ^ (uint32_t)(w[c] >> 32);
     if (acc == 0x12345u) sink[0] = acc;
-}
-
-// Packed fp32: fma.rn.f32x2 does two fused multiply-adds per instruction on a 64-bit register
-// pair.  WITH_WIDE == false: a pure chain (instructions per second); true: one wide multiply +
-// xor3 + one f32x2 per step, to compare with the same step carrying two scalar fmas.
-template <bool WITH_WIDE>
-__global__ void __launch_bounds__(kProbeThreads) probe_f32x2_kernel(int iters, uint32_t a, uint32_t b, uint32_t* sink) {
-    unsigned long long f[kChains], w[kChains];
-    const float fa = __uint_as_float(b), fb = 1e-7f;
-    unsigned long long aa, bb;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(aa) : "f"(fa), "f"(fa));
-    asm("mov.b64 %0, {%1, %2};" : "=l"(bb) : "f"(fb), "f"(fb));
-#pragma unroll
-    for (int c = 0; c < kChains; ++c) {
-        float x = 1.0f + 1e-3f * (float)(threadIdx.x + c), y = 1.0f - 1e-3f * (float)c;
-        asm("mov.b64 %0, {%1, %2};" : "=l"(f[c]) : "f"(x), "f"(y));
-        w[c] = ((unsigned long long)(threadIdx.x * 2654435761u + c * 40503u) << 32) | (blockIdx.x + 0x3f800001u + c);
-    }
-    for (int it = 0; it < iters; ++it) {
-#pragma unroll
-        for (int c = 0; c < kChains; ++c) {
-            if (WITH_WIDE) {
-                unsigned long long p;
-                asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(p) : "r"((uint32_t)w[c]), "r"(a));
-                w[c] = (uint32_t)(p >> 32) ^ (uint32_t)p ^ b;
-            }
-            asm volatile("fma.rn.f32x2 %0, %0, %1, %2;" : "+l"(f[c]) : "l"(aa), "l"(bb));
-        }
-    }
-    uint32_t acc = 0;
-#pragma unroll
-    for (int c = 0; c < kChains; ++c) acc ^= (uint32_t)f[c] ^ (uint32_t)(f[c] >> 32) ^ (uint32_t)w[c];
-    if (acc == 0x12345u) sink[0] = acc;
-}
-
-template <bool WITH_WIDE>
-int run_f32x2(int iters, uint32_t* sink, float* ms_out, double* ops_out) {
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return QES_ERR_CUDA;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return QES_ERR_CUDA;
-    cudaEvent_t e0, e1;
-    cudaEventCreate(&e0); cudaEventCreate(&e1);
-    int blocks = sms * kCtasPerSm;
-    probe_f32x2_kernel<WITH_WIDE><<<blocks, kProbeThreads>>>(iters / 8 + 1, 0xD2511F53u, 0x3f7ffff0u, sink);
-    cudaEventRecord(e0);
-    probe_f32x2_kernel<WITH_WIDE><<<blocks, kProbeThreads>>>(iters, 0xD2511F53u, 0x3f7ffff0u, sink);
-    cudaEventRecord(e1);
-    cudaError_t err = cudaEventSynchronize(e1);
-    float ms = 0.f;
-    cudaEventElapsedTime(&ms, e0, e1);
-    cudaEventDestroy(e0); cudaEventDestroy(e1);
-    if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return QES_ERR_CUDA;
-    *ms_out = ms;
-    *ops_out = (double)blocks * kProbeThreads * (double)iters * (double)kChains;   // f32x2 instructions, or steps
-    return QES_OK;
-}
-
-// The instruction mix of the update kernel with full instruction-level parallelism: per step
-// one wide multiply, 2.5 half-rate integer operations (the xor3 of the products plus 1.5
-// independent xor3) and two independent fp32 fused multiply-adds -- by the pipe rates 6 cycles
-// of the multiply pipe, 5 of the integer pipe, 5.5 issue slots.  What this kernel reaches is
-// what a schedule of that mix reaches on the machine.  ORDER sets the program order of the
-// instructions inside a step: 0 chain by chain, 1 kinds alternating, 2 kinds grouped.
-template <int ORDER>
-__global__ void __launch_bounds__(kProbeThreads) probe_mix_pass_kernel(int iters, uint32_t a, uint32_t b, uint32_t* sink) {
-    constexpr int kC = 4;
-    unsigned long long w[kC];
-    uint32_t u[kC], v[kC];
-    float f[kC][2];
-#pragma unroll
-    for (int c = 0; c < kC; ++c) {
-        w[c] = ((unsigned long long)(threadIdx.x * 2654435761u + c * 40503u) << 32) | (blockIdx.x + 0x3f800001u + c);
-        u[c] = threadIdx.x + 77u * c; v[c] = blockIdx.x + 13u * c;
-        f[c][0] = 1.0f + 1e-3f * (float)(threadIdx.x + c); f[c][1] = 1.0f - 1e-3f * (float)c;
-    }
-    const float fa = __uint_as_float(b), fb = 1e-7f;
-    for (int it = 0; it < iters; it += 2) {
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            if (ORDER == 0) {          // per chain: wide, its xor3, the independent xor3s, the two fmas
-#pragma unroll
-                for (int c = 0; c < kC; ++c) {
-                    unsigned long long p;
-                    asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(p) : "r"((uint32_t)w[c]), "r"(a));
-                    asm volatile("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(u[c]) : "r"(u[c]), "r"(a), "r"(b));
-                    uint32_t x;
-                    asm volatile("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(x) : "r"((uint32_t)(p >> 32)), "r"((uint32_t)p), "r"(b));
-                    w[c] = x;
-                    if (half == 0) asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(v[c]) : "r"(b), "r"(a));
-                    asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(f[c][0]) : "f"(fa), "f"(fb));
-                    asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(f[c][1]) : "f"(fa), "f"(fb));
-                }
-            } else if (ORDER == 1) {   // kinds alternate: wide, fma, xor3, fma, xor3 (+ xor3)
-                unsigned long long p[kC];
-#pragma unroll
-                for (int c = 0; c < kC; ++c) {
-                    asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(p[c]) : "r"((uint32_t)w[c]), "r"(a));
-                    asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(f[c][0]) : "f"(fa), "f"(fb));
-                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(u[c]) : "r"(a), "r"(b));
-                    asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(f[c][1]) : "f"(fa), "f"(fb));
-                    if (half == 0) asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(v[c]) : "r"(b), "r"(a));
-                    if (c > 0) {
-                        uint32_t x;
-                        asm volatile("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(x) : "r"((uint32_t)(p[c - 1] >> 32)), "r"((uint32_t)p[c - 1]), "r"(b));
-                        w[c - 1] = x;
-                    }
-                }
-                uint32_t x;
-                asm volatile("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(x) : "r"((uint32_t)(p[kC - 1] >> 32)), "r"((uint32_t)p[kC - 1]), "r"(b));
-                w[kC - 1] = x;
-            } else {                   // kinds grouped: all wides, all xor3s, all fmas
-                unsigned long long p[kC];
-#pragma unroll
-                for (int c = 0; c < kC; ++c) asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(p[c]) : "r"((uint32_t)w[c]), "r"(a));
-#pragma unroll
-                for (int c = 0; c < kC; ++c) {
-                    asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(u[c]) : "r"(a), "r"(b));
-                    if (half == 0) asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(v[c]) : "r"(b), "r"(a));
-                }
-#pragma unroll
-                for (int c = 0; c < kC; ++c) {
-                    uint32_t x;
-                    asm volatile("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(x) : "r"((uint32_t)(p[c] >> 32)), "r"((uint32_t)p[c]), "r"(b));
-                    w[c] = x;
-                }
-#pragma unroll
-                for (int c = 0; c < kC; ++c) {
-                    asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(f[c][0]) : "f"(fa), "f"(fb));
-                    asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(f[c][1]) : "f"(fa), "f"(fb));
-                }
-            }
-        }
-    }
-    uint32_t acc = 0;
-#pragma unroll
-    for (int c = 0; c < kC; ++c)
-        acc ^= (uint32_t)w[c] ^ (uint32_t)(w[c] >> 32) ^ u[c] ^ v[c] ^ __float_as_uint(f[c][0]) ^ __float_as_uint(f[c][1]);
-    if (acc == 0x12345u) sink[0] = acc;
-}
-
-template <int ORDER>
-int run_mix_pass(int iters, uint32_t* sink, float* ms_out, double* ops_out) {
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return QES_ERR_CUDA;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return QES_ERR_CUDA;
-    cudaEvent_t e0, e1;
-    cudaEventCreate(&e0); cudaEventCreate(&e1);
-    int blocks = sms * kCtasPerSm;
-    iters &= ~1;
-    probe_mix_pass_kernel<ORDER><<<blocks, kProbeThreads>>>(iters / 8 + 2, 0xD2511F53u, 0x3f7ffff0u, sink);
-    cudaEventRecord(e0);
-    probe_mix_pass_kernel<ORDER><<<blocks, kProbeThreads>>>(iters, 0xD2511F53u, 0x3f7ffff0u, sink);
-    cudaEventRecord(e1);
-    cudaError_t err = cudaEventSynchronize(e1);
-    float ms = 0.f;
-    cudaEventElapsedTime(&ms, e0, e1);
-    cudaEventDestroy(e0); cudaEventDestroy(e1);
-    if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return QES_ERR_CUDA;
-    *ms_out = ms;
-    *ops_out = (double)blocks * kProbeThreads * (double)iters * 4.0;   // steps (one wide multiply each)
-    return QES_OK;
 }
 
 template <int MODE>
@@ -347,28 +169,6 @@ int run_wide(int iters, uint32_t* sink, float* ms_out, double* ops_out) {
     if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return QES_ERR_CUDA;
     *ms_out = ms;
     *ops_out = (double)blocks * kProbeThreads * (double)iters * (double)kChains;   // steps, not instructions
-    return QES_OK;
-}
-
-template <int KA, int KB>
-int run_mix(int iters, uint32_t* sink, float* ms_out, double* ops_out) {
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return QES_ERR_CUDA;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return QES_ERR_CUDA;
-    cudaEvent_t e0, e1;
-    cudaEventCreate(&e0); cudaEventCreate(&e1);
-    int blocks = sms * kCtasPerSm;
-    probe_mix_kernel<KA, KB><<<blocks, kProbeThreads>>>(iters / 8 + 1, 0x9E3779B9u, 0x3f7ffff0u, sink);
-    cudaEventRecord(e0);
-    probe_mix_kernel<KA, KB><<<blocks, kProbeThreads>>>(iters, 0x9E3779B9u, 0x3f7ffff0u, sink);
-    cudaEventRecord(e1);
-    cudaError_t err = cudaEventSynchronize(e1);
-    float ms = 0.f;
-    cudaEventElapsedTime(&ms, e0, e1);
-    cudaEventDestroy(e0); cudaEventDestroy(e1);
-    if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return QES_ERR_CUDA;
-    *ms_out = ms;
-    *ops_out = (double)blocks * kProbeThreads * (double)iters * (double)kChains;
     return QES_OK;
 }
 
@@ -422,24 +222,10 @@ extern "C" int qes_pipe_probe(int32_t kind, int32_t iters, void* sink_dev, float
         case 17: return run_probe<17>(iters, sink, ms_out, ops_out);
         case 18: return run_wide<0>(iters, sink, ms_out, ops_out);
         case 19: return run_wide<1>(iters, sink, ms_out, ops_out);
-        case 20: return run_wide<2>(iters, sink, ms_out, ops_out);
-        case 21: return run_wide<3>(iters, sink, ms_out, ops_out);
-        case 22: return run_wide<4>(iters, sink, ms_out, ops_out);
-        case 23: return run_mix_pass<0>(iters, sink, ms_out, ops_out);
-        case 24: return run_mix_pass<1>(iters, sink, ms_out, ops_out);
-        case 25: return run_mix_pass<2>(iters, sink, ms_out, ops_out);
-        case 26: return run_f32x2<false>(iters, sink, ms_out, ops_out);
-        case 27: return run_f32x2<true>(iters, sink, ms_out, ops_out);
-        case 100: return run_mix<0, 1>(iters, sink, ms_out, ops_out);    // mul.wide + xor3
-        case 101: return run_mix<2, 1>(iters, sink, ms_out, ops_out);    // fma + xor3
-        case 102: return run_mix<0, 2>(iters, sink, ms_out, ops_out);    // mul.wide + fma
-        case 103: return run_mix<4, 1>(iters, sink, ms_out, ops_out);    // cvt + xor3
-        case 104: return run_mix<4, 0>(iters, sink, ms_out, ops_out);    // cvt + mul.wide
-        case 105: return run_mix<6, 9>(iters, sink, ms_out, ops_out);    // floor + rsqrt
-        case 106: return run_mix<6, 2>(iters, sink, ms_out, ops_out);    // floor + fma
-        case 107: return run_mix<10, 1>(iters, sink, ms_out, ops_out);   // add + xor3
-        case 108: return run_mix<12, 0>(iters, sink, ms_out, ops_out);   // fadd + mul.wide
-        case 109: return run_mix<14, 2>(iters, sink, ms_out, ops_out);   // compare/select + fma
+        case 20: return run_probe<20>(iters, sink, ms_out, ops_out);
+        case 21: return run_probe<21>(iters, sink, ms_out, ops_out);
+        case 22: return run_probe<22>(iters, sink, ms_out, ops_out);
+        case 23: return run_probe<23>(iters, sink, ms_out, ops_out);
         default: return QES_ERR_BAD_MODE;
     }
 }
