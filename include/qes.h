@@ -9,6 +9,8 @@
  *                        gate, repack — with Stateless Seed Replay     Algorithm 2; Eqs. 5-8
  *                        or with a stored residual                     Algorithm 1, update lines
  *   qes_replay_residual  the history loop of Algorithm 2 alone        Sec. 3.3
+ *   qes_gemv, qes_gemv_perturbed   the batch-1 weight read of a rollout, without and with the member's
+ *                        perturbation generated in the read              Algorithm 1, member loop
  *
  * Conventions shared by all entry points
  *  - Pointers named w*, scales*, seeds, fitness, residual*, stats are DEVICE pointers owned by the
@@ -184,6 +186,24 @@ int qes_estimate_bounds(float* eps_bound, float* rounding_bound, uint32_t* radiu
  */
 int qes_pair_deltas(const uint32_t* r0, const uint32_t* r1, const uint32_t* r2, const uint32_t* r3, int64_t n,
                     float sigma_eff, int8_t* delta_even, int8_t* delta_odd, uint8_t* verified, void* cuda_stream);
+
+/*
+ * The weight read of one decode step over a packed INT4 tensor: y[r] = sum_c scale[r, c / group] * q[r, c] * x[c]
+ * (batch 1; what a rollout's linear layer does with the weights the member loop of Algorithm 1 prepares).
+ *   qes_gemv            q = W as stored.
+ *   qes_gemv_perturbed  q = Gate(W + delta(seed, J)) (Eqs. 3-4; clamp mode: saturated), the member's perturbation
+ *                       regenerated inside the read instead of being stored by qes_perturb -- bit for bit the codes
+ *                       qes_perturb would write.  Uses sigma, sigma_unit, boundary_mode, antithetic of hparams;
+ *                       noise_mode must be QES_NOISE_PAIR24.
+ * desc: bits == 4, cols <= 102400; scales_f16 [device] is required (group_size > 0: [rows, cols / group_size];
+ * 0: [rows]); x_f16 [device, cols binary16 values, 16-byte aligned]; y [device, rows floats] is overwritten.
+ * Products are accumulated in binary16 over the 32 codes of a 128-bit word and in fp32 across words.
+ * These two calls exist to measure what perturbing on the fly costs against reading a stored perturbed copy.
+ */
+int qes_gemv(const qes_tensor_desc* desc, const void* w, const void* scales_f16, const void* x_f16, float* y,
+             void* cuda_stream);
+int qes_gemv_perturbed(const qes_tensor_desc* desc, const void* w, const void* scales_f16, uint64_t seed,
+                       const qes_hparams* hparams, const void* x_f16, float* y, void* cuda_stream);
 
 /*
  * Arithmetic-pipe throughput probes used to derive the ALU roofline (no counterpart in the

@@ -116,6 +116,10 @@ def load() -> C.CDLL:
         lib.qes_estimate_bounds.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_float), C.POINTER(C.c_uint32)]
         lib.qes_pair_deltas.restype = C.c_int
         lib.qes_pair_deltas.argtypes = [vp, vp, vp, vp, C.c_int64, C.c_float, vp, vp, vp, vp]
+        lib.qes_gemv.restype = C.c_int
+        lib.qes_gemv.argtypes = [C.POINTER(_TensorDesc), vp, vp, vp, vp, vp]
+        lib.qes_gemv_perturbed.restype = C.c_int
+        lib.qes_gemv_perturbed.argtypes = [C.POINTER(_TensorDesc), vp, vp, u64, C.POINTER(_HParams), vp, vp, vp]
         lib.qes_pipe_probe.restype = C.c_int
         lib.qes_pipe_probe.argtypes = [i32, i32, vp, C.POINTER(C.c_float), C.POINTER(C.c_double)]
         lib.qes_strerror.restype = C.c_char_p
@@ -220,6 +224,27 @@ def qes_gaussian_factors(r0, r1, radius, cosine, sine, stream=None) -> None:
                                      n, _ptr(radius, dtype=torch.float32, nbytes=4 * n, name="radius"),
                                      _ptr(cosine, dtype=torch.float32, nbytes=4 * n, name="cosine"),
                                      _ptr(sine, dtype=torch.float32, nbytes=4 * n, name="sine"), _stream(stream))
+    _check(rc)
+
+
+def qes_gemv(desc: TensorDesc, w, scales_f16, x_f16, y, stream=None) -> None:
+    """y = (scales * W) x for one packed INT4 tensor (batch 1, fp16 activations, fp32 result)."""
+    d = desc.c()
+    rc = load().qes_gemv(C.byref(d), _ptr(w, dtype=_W, nbytes=desc.packed_bytes, name="w"),
+                         _ptr(scales_f16, dtype=_S, nbytes=_scale_bytes(desc), name="scales"),
+                         _ptr(x_f16, dtype=torch.float16, nbytes=2 * desc.cols, name="x"),
+                         _ptr(y, dtype=torch.float32, nbytes=4 * desc.rows, name="y"), _stream(stream))
+    _check(rc)
+
+
+def qes_gemv_perturbed(desc: TensorDesc, w, scales_f16, seed: int, hparams: HParams, x_f16, y, stream=None) -> None:
+    """The same product over Gate(W + delta(seed)) with the perturbation generated inside the weight read."""
+    d, h = desc.c(), hparams.c()
+    rc = load().qes_gemv_perturbed(C.byref(d), _ptr(w, dtype=_W, nbytes=desc.packed_bytes, name="w"),
+                                   _ptr(scales_f16, dtype=_S, nbytes=_scale_bytes(desc), name="scales"),
+                                   C.c_uint64(seed & 0xFFFFFFFFFFFFFFFF), C.byref(h),
+                                   _ptr(x_f16, dtype=torch.float16, nbytes=2 * desc.cols, name="x"),
+                                   _ptr(y, dtype=torch.float32, nbytes=4 * desc.rows, name="y"), _stream(stream))
     _check(rc)
 
 

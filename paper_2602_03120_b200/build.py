@@ -5,7 +5,7 @@ import os
 import subprocess
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-SOURCES = [os.path.join(_HERE, "csrc", f) for f in ("qes_kernels.cu", "qes_probe.cu")]
+SOURCES = [os.path.join(_HERE, "csrc", f) for f in ("qes_kernels.cu", "qes_gemv.cu", "qes_probe.cu")]
 HEADERS = [os.path.join(_HERE, "csrc", "qes_device.cuh"),
            os.path.join(os.path.dirname(_HERE), "include", "qes.h")]
 LIB_PATH = os.path.join(_HERE, "libqes.so")

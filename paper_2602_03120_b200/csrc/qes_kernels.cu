@@ -6,8 +6,8 @@
 // contiguous 128 B / 256 B segment, once.  Everything else is arithmetic in registers: a code
 // costs one byte of HBM traffic but N*(K+1) noise samples of ~50 operations each, so the
 // kernels are bound by instruction issue on the multiply and integer pipes, never by memory;
-// kPairs is chosen for the register budget (S, e and the Philox state of 4 pairs fit without
-// spills at two CTAs per SM), not for the width of the load.
+// kPairs is chosen for the register budget (S, e and the Philox state of 4 pairs fit in 80
+// registers, three CTAs per SM, with a handful of spilled words), not for the width of the load.
 //
 // Per generation the CTA stages, in shared memory, the ten Philox round keys of each seed next
 // to the member's fitness and the seed's share of the first Philox rounds (96 B per seed,
@@ -25,7 +25,7 @@ enum PassMode : int { kStateless = 0, kStoredResidual = 1, kReplayOnly = 2 };
 
 constexpr int kThreads = 256;
 constexpr int kPairs = 4;
-constexpr int kMinBlocksPerSm = 2;
+constexpr int kMinBlocksPerSm = 3;   // 80 registers per thread: six warps per scheduler
 constexpr int kCodesPerThread = 2 * kPairs;
 constexpr int kSeedStride = 24;   // 32-bit words per staged member: a[10], b[10], fitness, SeedConst
 
