@@ -41,10 +41,33 @@ OPS_PER_SAMPLE_QUAD8 = (40 + 2 * 42 + 4 * 7) / 4.0
 OPS_PER_ELEM_GEN = 8.0      # u (2), round, w + step, two compares, select, residual
 OPS_PER_ELEM = 6.0          # unpack / repack
 SM_COUNT, LANES_PER_SM = 148, 128
-# DRAM bytes of one update launch per algorithmic byte (packed weights read once and written
-# once), from the ncu capture summarised under profiles/ (below 1: part of the last writes is
-# still in the 126 MB L2 when the kernel ends)
-DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE = 0.80
+# DRAM bytes of one update launch per algorithmic byte (packed weights read once and written once), from the
+# ncu capture of this kernel summarised in profiles/pass_kernel_int4_decoder1p5b_segment.md (below 1: part of
+# the last writes is still in the 126 MB L2 when the kernel ends).  None = the kernel has changed since the
+# counters were taken.
+DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE = None
+TRAFFIC_SOURCE = "scaled by codes from the one-launch ncu capture in profiles/pass_kernel_int4_decoder1p5b_segment.md"
+
+# Per-pipe form of the same roofline (default noise mode).  Scheduler cycles one warp instruction holds its pipe,
+# measured with qes_pipe_probe (profiles/pipe_probes_b200.md), and the instructions per noise sample that the
+# kernel's own path -- special-function estimate, verification, weighted sum -- needs on each pipe
+# (per Philox call = two samples: 20 wide multiplies and 20 xor3 by the definition of Philox4x32-10; fp32:
+# two multiplies each for radius and angle, the sigma scaling, two biased products, two offset removals, two
+# weighted-sum fmas = 11; integer pipe besides the xor3: uniform and angle conversions 3, two shift-adds,
+# two verifications, one radius-limit test, two top-byte additions = 10; special-function unit: lg2, sqrt,
+# sin, cos and the two floors = 6).
+PIPE_CYCLES = {"multiply_fp32": {"wide_multiply": 4.02, "fp32": 1.03}, "integer": {"int": 2.01}, "special_function": {"sfu": 8.0}}
+PIPE_OPS_PER_SAMPLE = {"multiply_fp32": {"wide_multiply": 10.0, "fp32": 5.5}, "integer": {"int": 15.0}, "special_function": {"sfu": 3.0}}
+
+
+def pipe_roofline(cycles_per_warp_sample: float):
+    """Each pipe's busy cycles per (warp, sample) at the measured rates, as a share of the measured cycles."""
+    pipes = {}
+    for pipe, kinds in PIPE_OPS_PER_SAMPLE.items():
+        busy = sum(n * PIPE_CYCLES[pipe][k] for k, n in kinds.items())
+        pipes[pipe] = {"ops_per_sample": sum(kinds.values()), "cycles_per_warp_sample": busy,
+                       "time_frac": busy / cycles_per_warp_sample}
+    return pipes
 
 
 def alu_ops(numel: int, n_pop: int, generations: int, per_sample: float = OPS_PER_SAMPLE) -> float:
@@ -358,12 +381,20 @@ def main():
     achieved = upd_ops_per_launch / upd_s_per_launch
     bytes_per_launch = 2 * wl.packed_bytes(cfg.bits, model.numel) * args.steps / n_upd_launches
     traffic = None if (DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE is None or quad or args.antithetic) else DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE * bytes_per_launch
+    # scheduler cycles per (warp, sample): launch time x clock x schedulers / warp-samples of the launch
+    warp_samples = model.numel * n_seeds * G * args.steps / n_upd_launches / 32.0
+    cycles_per_warp_sample = upd_s_per_launch * sm_mhz * 1e6 * SM_COUNT * 4 / warp_samples
+    pipes = None if quad else pipe_roofline(cycles_per_warp_sample)
     roofline = {"bound": "alu", "kernel": f"pass_kernel<{cfg.bits}> (qes_update, stateless)",
                 "achieved": achieved / 1e9, "peak": alu_peak / 1e9, "unit": "Glane-op/s", "frac": achieved / alu_peak,
                 "peak_source": f"{SM_COUNT} SMs x 4 schedulers x 32 lanes x {sm_mhz:.0f} MHz (one instruction per scheduler "
                                f"per cycle; SM clock from the {peak_src} peaks file)",
                 "ops_per_sample": per_sample, "avg_launch_ms": upd_s_per_launch * 1e3, "launches": n_upd_launches,
-                "traffic": traffic,
+                "traffic": traffic, "traffic_source": TRAFFIC_SOURCE if traffic is not None else None,
+                "cycles_per_warp_sample": cycles_per_warp_sample, "pipes": pipes,
+                "frac_pipe": None if pipes is None else max(v["time_frac"] for v in pipes.values()),
+                "pipe_source": "instruction mix of the kernel's own path per sample x cycles per warp instruction measured by "
+                               "qes_pipe_probe (profiles/pipe_probes_b200.md)",
                 "hbm": {"achieved_gbs": bytes_per_launch / upd_s_per_launch / 1e9, "peak_gbs": hbm_gbs,
                         "frac": bytes_per_launch / upd_s_per_launch / 1e9 / hbm_gbs, "of": peak_src}}
     line = {"metric": "weights_updated_per_s", "value": value, "unit": "weights/s", "n_gpus": world,

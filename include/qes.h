@@ -9,6 +9,7 @@
  *                        gate, repack — with Stateless Seed Replay     Algorithm 2; Eqs. 5-8
  *                        or with a stored residual                     Algorithm 1, update lines
  *   qes_replay_residual  the history loop of Algorithm 2 alone        Sec. 3.3
+ *   qes_replay_fidelity  gate-mismatch count of replay against a stored-residual run   Sec. 3.3
  *   qes_gemv, qes_gemv_perturbed   the batch-1 weight read of a rollout, without and with the member's
  *                        perturbation generated in the read              Algorithm 1, member loop
  *
@@ -144,6 +145,25 @@ int qes_replay_residual(const qes_tensor_desc* desc, const void* w, const void* 
 int qes_update(const qes_tensor_desc* desc, void* w_inout, const void* scales_f16,
                const uint64_t* seeds, const float* fitness, int32_t K, void* residual_inout,
                const qes_hparams* hparams, uint64_t* stats, void* cuda_stream);
+
+/*
+ * How faithfully Stateless Seed Replay reproduces a stored residual (Sec. 3.3: replay gates every past step
+ * against the current weights W_t instead of the weights W_tau of its own time; App. fidelity table).  For each
+ * element, in one launch: (1) Algorithm 1 with the residual kept, from e = 0 and the weights w_start, over the
+ * `generations` rows of the table (oldest first), the weights moving and each step gated against the weights of
+ * its time; (2) Algorithm 2's history loop over the same rows from e = 0, gated against the FINAL weights of (1).
+ *   counts [device, 4 x uint64, ADDED to (caller zeroes)]: [0] elements whose per-generation records of blocked
+ *          (or, in clamp mode, shortened) steps differ between (1) and (2) -- the gate-mismatch count;
+ *          [1] elements with at least one blocked step in (1); [2] elements whose final residuals differ by more
+ *          than 1e-5 (with the gate a subset of [0]: equal records give bit-equal residuals; a clamp can shorten the same
+ *          step by different amounts in the two runs); [3] elements whose code moved.
+ *   w_end_out [device, nullable] receives the final weights of (1); may alias w_start exactly.
+ * seeds / fitness as for qes_replay_residual with K = generations, 1 <= generations <= 64; noise_mode must be
+ * QES_NOISE_PAIR24.  Costs two noise passes; a diagnostic, not part of the training step.
+ */
+int qes_replay_fidelity(const qes_tensor_desc* desc, const void* w_start, void* w_end_out, const void* scales_f16,
+                        const uint64_t* seeds, const float* fitness, int32_t generations, const qes_hparams* hparams,
+                        uint64_t* counts, void* cuda_stream);
 
 /*
  * The Box-Muller factors of the noise contract on their own (Sec. 3.2 "RNG(seed)"; the paper

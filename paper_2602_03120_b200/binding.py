@@ -116,6 +116,8 @@ def load() -> C.CDLL:
         lib.qes_estimate_bounds.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_float), C.POINTER(C.c_uint32)]
         lib.qes_pair_deltas.restype = C.c_int
         lib.qes_pair_deltas.argtypes = [vp, vp, vp, vp, C.c_int64, C.c_float, vp, vp, vp, vp]
+        lib.qes_replay_fidelity.restype = C.c_int
+        lib.qes_replay_fidelity.argtypes = [C.POINTER(_TensorDesc), vp, vp, vp, vp, vp, i32, C.POINTER(_HParams), vp, vp]
         lib.qes_gemv.restype = C.c_int
         lib.qes_gemv.argtypes = [C.POINTER(_TensorDesc), vp, vp, vp, vp, vp]
         lib.qes_gemv_perturbed.restype = C.c_int
@@ -224,6 +226,20 @@ def qes_gaussian_factors(r0, r1, radius, cosine, sine, stream=None) -> None:
                                      n, _ptr(radius, dtype=torch.float32, nbytes=4 * n, name="radius"),
                                      _ptr(cosine, dtype=torch.float32, nbytes=4 * n, name="cosine"),
                                      _ptr(sine, dtype=torch.float32, nbytes=4 * n, name="sine"), _stream(stream))
+    _check(rc)
+
+
+def qes_replay_fidelity(desc: TensorDesc, w_start, w_end_out, scales_f16, seeds, fitness, generations: int,
+                        hparams: HParams, counts, stream=None) -> None:
+    """Gate-mismatch count of Stateless Seed Replay against a stored-residual run over `generations` steps (Sec. 3.3)."""
+    d, h = desc.c(), hparams.c()
+    n, ns = generations * hparams.n_pop, generations * hparams.seeds_per_generation
+    rc = load().qes_replay_fidelity(C.byref(d), _ptr(w_start, dtype=_W, nbytes=desc.packed_bytes, name="w_start"),
+                                    _ptr(w_end_out, dtype=_W, nbytes=desc.packed_bytes, name="w_end_out"),
+                                    _ptr(scales_f16, dtype=_S, nbytes=_scale_bytes(desc), name="scales"),
+                                    _ptr(seeds, dtype=_SEEDS, nbytes=8 * ns, name="seeds"),
+                                    _ptr(fitness, dtype=torch.float32, nbytes=4 * n, name="fitness"), generations, C.byref(h),
+                                    _ptr(counts, dtype=_SEEDS, nbytes=32, name="counts"), _stream(stream))
     _check(rc)
 
 

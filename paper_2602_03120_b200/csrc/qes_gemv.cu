@@ -63,7 +63,7 @@ __device__ __forceinline__ uint32_t perturbed_word(uint32_t w, uint32_t call_lo,
         uint32_t r0, r1, r2, r3;
         philox_tail(make_pair_const(call_lo + i), sc, rk, r0, r1, r2, r3);
         int z[2];
-        if (pair_rounding_sums_estimate<CLAMP_DELTA>(r0, r1, r2, r3, nsig24, guard, z[0], z[1]))
+        if (pair_rounding_sums_estimate<CLAMP_DELTA, false>(r0, r1, r2, r3, nsig24, guard, z[0], z[1]))
             call_rounding_sums<CLAMP_DELTA, false>(r0, r1, r2, r3, nsig24, z);
 #pragma unroll
         for (int j = 0; j < 2; ++j) {

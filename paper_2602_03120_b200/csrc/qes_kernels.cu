@@ -153,20 +153,15 @@ __global__ void __launch_bounds__(kThreads) perturb_kernel(PassParams p, RoundKe
     Chunk<BITS, kPairs> out, out_minus;
     out.clear();
     out_minus.clear();
-    FastGuard guard;
-    if constexpr (!QUAD) guard = make_fast_guard(nsig24);
+    const FastGuard guard = make_fast_guard(nsig24);
 #pragma unroll
     for (int i = 0; i < kCalls; ++i) {
         uint32_t r0, r1, r2, r3;
         philox_tail(make_pair_const(x0 + i), sc, rk, r0, r1, r2, r3);
         int z[kPerCall];
-        if constexpr (QUAD) {
-            call_rounding_sums<CLAMP_DELTA, true>(r0, r1, r2, r3, nsig24, z);
-        } else {
-            // special-function estimate first; the exact sequence only where the estimate cannot decide
-            if (pair_rounding_sums_estimate<CLAMP_DELTA>(r0, r1, r2, r3, nsig24, guard, z[0], z[1]))
-                call_rounding_sums<CLAMP_DELTA, false>(r0, r1, r2, r3, nsig24, z);
-        }
+        // special-function estimate first; the exact sequence only where the estimate cannot decide
+        if (call_rounding_sums_estimate<CLAMP_DELTA, QUAD>(r0, r1, r2, r3, nsig24, guard, z))
+            call_rounding_sums<CLAMP_DELTA, QUAD>(r0, r1, r2, r3, nsig24, z);
 #pragma unroll
         for (int j = 0; j < kPerCall; ++j) {
             const int t = kPerCall * i + j;
@@ -214,6 +209,53 @@ __device__ __forceinline__ RoundKeys load_round_keys(const uint32_t* entry, floa
     return rk;
 }
 
+// Eq. 5's numerator for one generation: S[t] = sum_i F_i * delta_i for the thread's T codes, the seeds' staged
+// entries read in member order (the same order in every thread: each read is a broadcast).
+template <bool CLAMP_DELTA, bool QUAD>
+__device__ __forceinline__ void generation_sums(const uint32_t* table, int n_seeds, const PairConst (&pc)[kCodesPerThread / (QUAD ? 4 : 2)],
+                                                uint32_t y, bool y_uniform, float nsig24, const FastGuard& guard, int nd_max,
+                                                float (&S)[kCodesPerThread]) {
+    constexpr int T = kCodesPerThread;
+    constexpr int kPerCall = QUAD ? 4 : 2;
+    constexpr int kCalls = T / kPerCall;
+#pragma unroll
+    for (int t = 0; t < T; ++t) S[t] = 0.0f;
+#pragma unroll 1
+    for (int i = 0; i < n_seeds; ++i) {
+        float Fm;   // -F_i
+        SeedConst sc;
+        const RoundKeys rk = load_round_keys(table + i * kSeedStride, Fm, sc);
+        if (!y_uniform) sc = make_seed_const(y, rk);
+        float nd[T];   // -delta of this seed for the thread's codes
+        // special-function estimates for all of the thread's samples of this seed; if any of the eight lies
+        // too close to a rounding decision for the estimate to settle it (about 1.5e-4 of the (thread, seed)
+        // steps at sigma = 0.5), the seed is redone with the exact sequence
+        bool undecided = false;
+#pragma unroll
+        for (int c = 0; c < kCalls; ++c) {
+            uint32_t r0, r1, r2, r3;
+            philox_tail(pc[c], sc, rk, r0, r1, r2, r3);
+            int z[kPerCall];
+            undecided |= call_rounding_sums_estimate<CLAMP_DELTA, QUAD>(r0, r1, r2, r3, nsig24, guard, z);
+#pragma unroll
+            for (int j = 0; j < kPerCall; ++j) nd[kPerCall * c + j] = neg_delta_float<CLAMP_DELTA>(z[j], nd_max);
+        }
+        if (__builtin_expect(undecided, 0)) {
+#pragma unroll
+            for (int c = 0; c < kCalls; ++c) {
+                uint32_t r0, r1, r2, r3;
+                philox_tail(pc[c], sc, rk, r0, r1, r2, r3);
+                int z[kPerCall];
+                call_rounding_sums<CLAMP_DELTA, QUAD>(r0, r1, r2, r3, nsig24, z);
+#pragma unroll
+                for (int j = 0; j < kPerCall; ++j) nd[kPerCall * c + j] = neg_delta_float<CLAMP_DELTA>(z[j], nd_max);
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < T; ++t) S[t] = fmaf(Fm, nd[t], S[t]);      // Eq. 5 numerator
+    }
+}
+
 // Algorithm 2 (stateless), Algorithm 1's update lines (stored residual) or the history loop
 // alone (replay only), selected by p.mode.  Shared memory: 2 * (seeds per generation) * 96 B.
 template <int BITS, bool CLAMP_DELTA, bool STATS, bool QUAD>
@@ -244,8 +286,7 @@ __global__ void __launch_bounds__(kThreads, kMinBlocksPerSm) pass_kernel(PassPar
         for (int i = 0; i < kCalls; ++i) pc[i] = make_pair_const((uint32_t)call0 + i);
     }
 
-    FastGuard guard;
-    if constexpr (!QUAD) guard = make_fast_guard(nsig24);
+    const FastGuard guard = make_fast_guard(nsig24);
 
     const int last = p.generations - 1;
     const int buf_words = p.n_seeds * kSeedStride;
@@ -269,54 +310,7 @@ __global__ void __launch_bounds__(kThreads, kMinBlocksPerSm) pass_kernel(PassPar
         if (!active) continue;
         const uint32_t* table = smem + (k & 1) * buf_words;
         float S[T];
-#pragma unroll
-        for (int t = 0; t < T; ++t) S[t] = 0.0f;
-#pragma unroll 1
-        for (int i = 0; i < p.n_seeds; ++i) {
-            float Fm;   // -F_i
-            SeedConst sc;
-            const RoundKeys rk = load_round_keys(table + i * kSeedStride, Fm, sc);
-            if (!y_uniform) sc = make_seed_const(y, rk);
-            float nd[T];   // -delta of this seed for the thread's codes
-            if constexpr (QUAD) {
-#pragma unroll
-                for (int c = 0; c < kCalls; ++c) {
-                    uint32_t r0, r1, r2, r3;
-                    philox_tail(pc[c], sc, rk, r0, r1, r2, r3);
-                    int z[kPerCall];
-                    call_rounding_sums<CLAMP_DELTA, true>(r0, r1, r2, r3, nsig24, z);
-#pragma unroll
-                    for (int j = 0; j < kPerCall; ++j) nd[kPerCall * c + j] = neg_delta_float<CLAMP_DELTA>(z[j], p.nd_max);
-                }
-            } else {
-                // special-function estimates for all four pairs; if any of the eight samples lies too
-                // close to a rounding decision for the estimate to settle it (about 1.5e-4 of the
-                // (thread, seed) steps at sigma = 0.5), the seed is redone with the exact sequence
-                bool undecided = false;
-#pragma unroll
-                for (int c = 0; c < kCalls; ++c) {
-                    uint32_t r0, r1, r2, r3;
-                    philox_tail(pc[c], sc, rk, r0, r1, r2, r3);
-                    int ze, zo;
-                    undecided |= pair_rounding_sums_estimate<CLAMP_DELTA>(r0, r1, r2, r3, nsig24, guard, ze, zo);
-                    nd[2 * c] = neg_delta_float<CLAMP_DELTA>(ze, p.nd_max);
-                    nd[2 * c + 1] = neg_delta_float<CLAMP_DELTA>(zo, p.nd_max);
-                }
-                if (__builtin_expect(undecided, 0)) {
-#pragma unroll
-                    for (int c = 0; c < kCalls; ++c) {
-                        uint32_t r0, r1, r2, r3;
-                        philox_tail(pc[c], sc, rk, r0, r1, r2, r3);
-                        int z[2];
-                        call_rounding_sums<CLAMP_DELTA, false>(r0, r1, r2, r3, nsig24, z);
-                        nd[2 * c] = neg_delta_float<CLAMP_DELTA>(z[0], p.nd_max);
-                        nd[2 * c + 1] = neg_delta_float<CLAMP_DELTA>(z[1], p.nd_max);
-                    }
-                }
-            }
-#pragma unroll
-            for (int t = 0; t < T; ++t) S[t] = fmaf(Fm, nd[t], S[t]);      // Eq. 5 numerator
-        }
+        generation_sums<CLAMP_DELTA, QUAD>(table, p.n_seeds, pc, y, y_uniform, nsig24, guard, p.nd_max, S);
         const bool is_update = (k == last) && (p.mode != kReplayOnly);
 #pragma unroll
         for (int t = 0; t < T; ++t) {
@@ -358,6 +352,103 @@ __global__ void __launch_bounds__(kThreads, kMinBlocksPerSm) pass_kernel(PassPar
     }
 }
 
+// Sec. 3.3 measured on a true trajectory.  Pass 0: Algorithm 1 with the residual kept (here: in registers) over the
+// table's generations, starting from e = 0 and the given weights, each step gated against the weights of its own
+// time.  Pass 1: Algorithm 2's history loop over the same generations, gated against the FINAL weights, as a
+// stateless update at that point would replay them.  Counted per element: the two records of blocked steps
+// differ; any step was blocked on the true trajectory; the two final residuals differ; the code moved.
+template <int BITS, bool CLAMP_DELTA>
+__global__ void __launch_bounds__(kThreads) fidelity_kernel(PassParams p) {
+    extern __shared__ __align__(16) uint32_t smem[];
+    constexpr int T = kCodesPerThread;
+    constexpr int kCalls = T / 2;
+    const int64_t chunk = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const bool active = chunk < p.n_chunks;
+    Chunk<BITS, kPairs> w;
+    w.clear();
+    float nsig24 = 0.0f;
+    PairConst pc[kCalls];
+    uint32_t y = 0u;
+    if (active) {
+        w.load(p.w_in, chunk);
+        nsig24 = chunk_neg_sigma24(p, chunk);
+        const uint64_t call0 = (p.elem_offset >> 1) + (uint64_t)chunk * kCalls;
+        y = (uint32_t)(call0 >> 32);
+#pragma unroll
+        for (int i = 0; i < kCalls; ++i) pc[i] = make_pair_const((uint32_t)call0 + i);
+    }
+    const FastGuard guard = make_fast_guard(nsig24);
+    const uint64_t cta_call0 = (p.elem_offset >> 1) + (uint64_t)blockIdx.x * (kThreads * kCalls);
+    const uint32_t y_cta = (uint32_t)(cta_call0 >> 32);
+    const bool y_uniform = (uint32_t)((cta_call0 + (uint64_t)(kThreads * kCalls - 1)) >> 32) == y_cta;
+    const int buf_words = p.n_seeds * kSeedStride;
+    const int fit_per_gen = p.antithetic ? 2 * p.n_seeds : p.n_seeds;
+
+    float wcur[T], e[T], e_true[T];
+    unsigned long long blocked_true[T], blocked_replay[T];
+#pragma unroll
+    for (int t = 0; t < T; ++t) {
+        wcur[t] = (float)w.get(t);
+        e[t] = 0.0f; e_true[t] = 0.0f;
+        blocked_true[t] = 0ull; blocked_replay[t] = 0ull;
+    }
+    for (int pass = 0; pass < 2; ++pass) {
+        __syncthreads();   // nobody still reads the staging buffers of the previous pass
+        stage_generation(smem, p.seeds, p.fitness, p.n_seeds, p.antithetic != 0, y_cta);
+        for (int k = 0; k < p.generations; ++k) {
+            __syncthreads();
+            if (k + 1 < p.generations)
+                stage_generation(smem + ((k + 1) & 1) * buf_words, p.seeds + (int64_t)(k + 1) * p.n_seeds,
+                                 p.fitness + (int64_t)(k + 1) * fit_per_gen, p.n_seeds, p.antithetic != 0, y_cta);
+            if (!active) continue;
+            float S[T];
+            generation_sums<CLAMP_DELTA, false>(smem + (k & 1) * buf_words, p.n_seeds, pc, y, y_uniform, nsig24, guard, p.nd_max, S);
+#pragma unroll
+            for (int t = 0; t < T; ++t) {
+                const float u = fmaf(p.coef, S[t], p.gamma * e[t]);                        // Eq. 6
+                const float step = roundf(u);                                               // Eq. 7
+                const float applied = applied_step(wcur[t], step, p.qmin, p.qmax, p.boundary_mode);
+                e[t] = u - applied;                                                         // Eq. 8
+                const unsigned long long bit = applied != step ? 1ull << k : 0ull;
+                if (pass == 0) {
+                    blocked_true[t] |= bit;
+                    wcur[t] += applied;            // the weights move: the next step is gated against W_{tau+1}
+                } else {
+                    blocked_replay[t] |= bit;      // wcur stays at the final weights
+                }
+            }
+        }
+        if (pass == 0) {
+#pragma unroll
+            for (int t = 0; t < T; ++t) { e_true[t] = e[t]; e[t] = 0.0f; }
+        }
+    }
+    unsigned int n_mismatch = 0, n_blocked = 0, n_residual = 0, n_moved = 0;
+    if (active) {
+        Chunk<BITS, kPairs> out;
+        out.clear();
+#pragma unroll
+        for (int t = 0; t < T; ++t) {
+            n_mismatch += blocked_true[t] != blocked_replay[t];
+            n_blocked += blocked_true[t] != 0ull;
+            n_residual += fabsf(e[t] - e_true[t]) > 1e-5f;
+            n_moved += wcur[t] != (float)w.get(t);
+            out.put(t, (int)wcur[t]);
+        }
+        if (p.w_out != nullptr) out.store(p.w_out, chunk);
+    }
+    n_mismatch = __reduce_add_sync(0xffffffffu, n_mismatch);
+    n_blocked = __reduce_add_sync(0xffffffffu, n_blocked);
+    n_residual = __reduce_add_sync(0xffffffffu, n_residual);
+    n_moved = __reduce_add_sync(0xffffffffu, n_moved);
+    if ((threadIdx.x & 31) == 0) {
+        if (n_mismatch) atomicAdd(p.stats + 0, (unsigned long long)n_mismatch);
+        if (n_blocked) atomicAdd(p.stats + 1, (unsigned long long)n_blocked);
+        if (n_residual) atomicAdd(p.stats + 2, (unsigned long long)n_residual);
+        if (n_moved) atomicAdd(p.stats + 3, (unsigned long long)n_moved);
+    }
+}
+
 // Box-Muller factors of word pairs, for checking the frozen fp32 sequence on its whole domain.
 __global__ void __launch_bounds__(kThreads) gaussian_factors_kernel(const uint32_t* r0, const uint32_t* r1, int64_t n,
                                                                     float* R, float* C, float* S) {
@@ -393,7 +484,7 @@ __global__ void __launch_bounds__(kThreads) pair_deltas_kernel(const uint32_t* r
     if (i >= n) return;
     const FastGuard guard = make_fast_guard(nsig24);
     int z[2];
-    const bool undecided = pair_rounding_sums_estimate<true>(r0[i], r1[i], r2[i], r3[i], nsig24, guard, z[0], z[1]);
+    const bool undecided = pair_rounding_sums_estimate<true, false>(r0[i], r1[i], r2[i], r3[i], nsig24, guard, z[0], z[1]);
     if (undecided) call_rounding_sums<true, false>(r0[i], r1[i], r2[i], r3[i], nsig24, z);
     d_even[i] = (signed char)(-neg_delta<true>(z[0], 8));
     d_odd[i] = (signed char)(-neg_delta<true>(z[1], 8));
@@ -606,6 +697,41 @@ int qes_update(const qes_tensor_desc* desc, void* w_inout, const void* scales_f1
     p.mode = residual_inout != nullptr ? kStoredResidual : kStateless;
     return dispatch_pass(desc->bits, delta_clamp_needed(hparams), hparams->noise_mode == QES_NOISE_QUAD8, p,
                          reinterpret_cast<cudaStream_t>(cuda_stream));
+}
+
+int qes_replay_fidelity(const qes_tensor_desc* desc, const void* w_start, void* w_end_out, const void* scales_f16,
+                        const uint64_t* seeds, const float* fitness, int32_t generations, const qes_hparams* hparams,
+                        uint64_t* counts, void* cuda_stream) {
+    int rc = validate(desc, hparams);
+    if (rc != QES_OK) return rc;
+    if (generations < 1 || generations > 64) return QES_ERR_BAD_HPARAM;
+    if (hparams->noise_mode != QES_NOISE_PAIR24) return QES_ERR_BAD_MODE;
+    if (w_start == nullptr || counts == nullptr) return QES_ERR_NULL_PTR;
+    if (hparams->sigma_unit == QES_SIGMA_WEIGHT && scales_f16 == nullptr) return QES_ERR_NULL_PTR;
+    if (!aligned(w_start, 16) || !aligned(w_end_out, 16) || !aligned(scales_f16, 2) || !aligned(counts, 8)) return QES_ERR_MISALIGNED;
+    rc = check_table(seeds, fitness, generations, hparams);
+    if (rc != QES_OK) return rc;
+    PassParams p = base_params(desc, hparams, scales_f16);
+    p.w_in = w_start;
+    p.w_out = w_end_out;
+    p.seeds = seeds;
+    p.fitness = fitness;
+    p.stats = reinterpret_cast<unsigned long long*>(counts);
+    p.generations = generations;
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    const size_t smem = stage_bytes(p.n_seeds);
+    const unsigned blocks = (unsigned)((p.n_chunks + kThreads - 1) / kThreads);
+    auto launch = [&](auto kernel) {
+        if (smem > 48 * 1024 && cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+            cudaGetLastError();
+            return (int)QES_ERR_CUDA;
+        }
+        kernel<<<blocks, kThreads, smem, stream>>>(p);
+        return cudaGetLastError() == cudaSuccess ? (int)QES_OK : (int)QES_ERR_CUDA;
+    };
+    const bool clamp = delta_clamp_needed(hparams);
+    if (desc->bits == 4) return clamp ? launch(fidelity_kernel<4, true>) : launch(fidelity_kernel<4, false>);
+    return clamp ? launch(fidelity_kernel<8, true>) : launch(fidelity_kernel<8, false>);
 }
 
 int qes_gaussian_factors(const uint32_t* r0, const uint32_t* r1, int64_t n, float* radius, float* cosine,

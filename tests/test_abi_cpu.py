@@ -34,7 +34,8 @@ def test_every_declared_symbol_is_exported(lib):
     header = open(os.path.join(ROOT, "include", "qes.h")).read()
     names = re.findall(r"^(?:int|const char\*)\s+(qes_\w+)\s*\(", header, flags=re.M)
     assert set(names) >= {"qes_perturb", "qes_update", "qes_replay_residual", "qes_perturb_pair", "qes_gaussian_factors", "qes_pipe_probe",
-                          "qes_gaussian_estimates", "qes_estimate_bounds", "qes_pair_deltas", "qes_strerror", "qes_version"}
+                          "qes_gaussian_estimates", "qes_estimate_bounds", "qes_pair_deltas", "qes_gemv", "qes_gemv_perturbed",
+                          "qes_replay_fidelity", "qes_strerror", "qes_version"}
     for n in names:
         assert hasattr(lib, n), n
     assert lib.qes_version() >= 100
@@ -95,6 +96,16 @@ def test_invalid_arguments_are_rejected_without_launching(lib):
     assert lib.qes_pair_deltas(0x1000, 0x2000, 0x3000, 0x4000, 8, C.c_float(0.0), 0x5000, 0x6000, None, None) == -5
     assert lib.qes_pair_deltas(0x1000, 0x2000, 0x3000, None, 8, C.c_float(0.5), 0x5000, 0x6000, None, None) == -1
     assert lib.qes_estimate_bounds(None, None, None) == -1
+    assert lib.qes_replay_fidelity(C.byref(d), 0x1000, None, None, 0x2000, 0x3000, 0, C.byref(h), 0x7000, None) == -5
+    assert lib.qes_replay_fidelity(C.byref(d), 0x1000, None, None, 0x2000, 0x3000, 65, C.byref(h), 0x7000, None) == -5
+    assert lib.qes_replay_fidelity(C.byref(d), 0x1000, None, None, 0x2000, 0x3000, 4, C.byref(h), None, None) == -1
+    assert lib.qes_replay_fidelity(C.byref(d), 0x1000, 0x5008, None, 0x2000, 0x3000, 4, C.byref(h), 0x7000, None) == -4
+    assert lib.qes_gemv(C.byref(d), 0x1000, None, 0x2000, 0x3000, None) == -1
+    assert lib.qes_gemv(C.byref(d), 0x1000, 0x4000, 0x2008, 0x3000, None) == -4
+    d8 = binding.TensorDesc(bits=8, rows=4, cols=64).c()
+    assert lib.qes_gemv(C.byref(d8), 0x1000, 0x4000, 0x2000, 0x3000, None) == -2
+    assert lib.qes_gemv_perturbed(C.byref(d), 0x1000, 0x4000, 1, None, 0x2000, 0x3000, None) == -1
+    assert lib.qes_gemv_perturbed(C.byref(d), 0x1000, 0x4000, 1, C.byref(h5), 0x2000, 0x3000, None) == -6
     eps, rnd, lim = binding.qes_estimate_bounds()
     assert 0 < eps < 1e-4 and 0 < rnd < 1e-5 and lim > 0xFF000000
     for code in range(-8, 1):

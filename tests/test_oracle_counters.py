@@ -6,6 +6,7 @@ import numpy as np
 import pytest
 
 from paper_2602_03120_b200 import workloads as wl
+from stored_trajectory import stored_trajectory
 
 
 def _tensor(qo, codes, bits=4, cols=None, **kw):
@@ -82,26 +83,6 @@ def test_counters_with_the_blocked_signal_carried(qo):
     assert replay.max() >= 3 and np.abs(e).max() >= 4          # carried signal grows past one step
 
 
-def _stored_trajectory(qo, t, codes, seeds, fit, hp, bits):
-    """Algorithm 1 step by step with the residual kept (in double): codes, residual and the record of
-    blocked steps (bit s = step s) as they really happened against the evolving weights."""
-    n = codes.size
-    cur, e, mask = qo.pack(bits, codes), np.zeros(n), np.zeros(n, np.uint64)
-    J = np.arange(n, dtype=np.uint64) + np.uint64(t.elem_offset)
-    c = float(np.float32(hp.lr)) / (hp.n_pop * float(np.float32(hp.sigma)))
-    for s in range(seeds.shape[0]):
-        W = qo.unpack(bits, cur, n).astype(np.int64)
-        S = sum(float(fit[s, i]) * qo.delta(int(seeds[s, i]), J, hp.sigma)[0] for i in range(hp.n_pop))
-        u = c * S + float(np.float32(hp.gamma)) * e
-        step = (np.sign(u) * np.floor(np.abs(u) + 0.5)).astype(np.int64)
-        ok = (W + step >= t.c().qmin) & (W + step <= t.c().qmax)
-        applied = np.where(ok, step, 0)
-        mask |= (~ok).astype(np.uint64) << np.uint64(s)
-        e = u - applied
-        cur = qo.pack(bits, (W + applied).astype(np.int32))
-    return cur, e, mask
-
-
 def test_gate_mismatch_count_on_a_true_trajectory_with_a_firing_gate(qo):
     """Sec. 3.3: replay gates against the current weights W_t, the stored-residual run gated against
     W_tau.  INT4 uniform codes, T = 6 steps: the two records of blocked steps differ on a counted set of
@@ -111,7 +92,7 @@ def test_gate_mismatch_count_on_a_true_trajectory_with_a_firing_gate(qo):
     t, _ = _tensor(qo, codes, cols=256, elem_offset=1 << 16)
     hp = qo.HParams(sigma=0.5, lr=1.0, gamma=0.9, n_pop=N)
     seeds, fit = wl.draw_seeds(T, N, stream=41), wl.draw_fitness(T, N, stream=41)
-    cur, e_stored, mask_stored = _stored_trajectory(qo, t, codes, seeds, fit, hp, 4)
+    cur, e_stored, mask_stored, _ = stored_trajectory(qo, t, codes, seeds, fit, hp, 4)
     rep = qo.replay_residual(t, cur, None, seeds, fit, T, hp)
     agree = rep["blocked"] == mask_stored
     mismatches = int((~agree).sum())
@@ -123,7 +104,7 @@ def test_gate_mismatch_count_on_a_true_trajectory_with_a_firing_gate(qo):
     assert np.all(np.abs(rep["e"][~agree] - e_stored[~agree]) > 1e-3)
     # with a range the walk cannot reach, nothing is ever blocked and the two runs agree everywhere
     t8, _ = _tensor(qo, codes, bits=8, cols=256, elem_offset=1 << 16)
-    cur8, e8, m8 = _stored_trajectory(qo, t8, codes, seeds, fit, hp, 8)
+    cur8, e8, m8, _ = stored_trajectory(qo, t8, codes, seeds, fit, hp, 8)
     rep8 = qo.replay_residual(t8, cur8, None, seeds, fit, T, hp)
     assert not m8.any() and not rep8["blocked"].any() and np.allclose(rep8["e"], e8, atol=1e-12)
 
