@@ -45,7 +45,7 @@ SM_COUNT, LANES_PER_SM = 148, 128
 # ncu capture of this kernel summarised in profiles/pass_kernel_int4_decoder1p5b_segment.md (below 1: part of
 # the last writes is still in the 126 MB L2 when the kernel ends).  None = the kernel has changed since the
 # counters were taken.
-DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE = None
+DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE = 0.80
 TRAFFIC_SOURCE = "scaled by codes from the one-launch ncu capture in profiles/pass_kernel_int4_decoder1p5b_segment.md"
 
 # Per-pipe form of the same roofline (default noise mode).  Scheduler cycles one warp instruction holds its pipe,
