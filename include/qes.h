@@ -33,7 +33,7 @@
  *  - The kernels first estimate each noise sample with the GPU's special-function unit and recompute
  *    it with the exact fp32 sequence of the contract only where the estimate cannot settle Eq. 3's
  *    rounding decision; results are identical to computing every sample exactly.
- *  - Fitness values are the already normalised rewards F_i (Algorithm 1, "Normalize reward").
+ *  - Fitness values are the already normalised rewards F_i (Algorithm 1, the reward-normalisation line).
  *  - Return value: QES_OK, or a negative qes_status; on any error nothing was launched and no
  *    buffer was touched.
  */

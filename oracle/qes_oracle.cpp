@@ -228,7 +228,7 @@ struct Tensor { int32_t bits, qmin, qmax, group_size; int64_t rows, cols; uint64
 // antithetic != 0 (App. A "antithetic perturbation pairs"): the population is n_pop / 2 pairs, pair j
 // has one seed and the two members W + delta_j and W - delta_j; seeds hold n_pop / 2 entries per
 // generation, fitness holds n_pop entries per generation ordered F+_0, F-_0, F+_1, F-_1, ...
-// residual_f16 != 0: the stored residual of Algorithm 1 is kept in binary16 ("Residuals e_0 <- 0 (FP16)"):
+// residual_f16 != 0: the stored residual of Algorithm 1 is kept in binary16 (the precision its initialisation line gives the residual):
 // read as binary16, all arithmetic as before; the caller rounds the returned e back to binary16.
 struct HParams { float sigma, lr, gamma; int32_t n_pop, sigma_unit, boundary_mode, antithetic, residual_f16, noise_mode; };
 
@@ -393,7 +393,7 @@ long long qo_applied_step(int w, long long step, int qmin, int qmax, int mode) {
     return applied_step(w, step, qmin, qmax, mode);
 }
 
-// Algorithm 1, lines "Reconstruct delta_i" and "Gate(W + delta_i)" for one member.
+// Algorithm 1, member loop: the member's perturbation rebuilt from its seed and applied under the gate.
 // idx == NULL: elements 0..n-1.  w_out[i] = perturbed code of element idx[i].
 // sign = +1: W + delta; sign = -1: the antithetic member W - delta (App. A).
 int qo_perturb(const Tensor* t, const uint8_t* w, const uint16_t* scales, uint64_t seed, int sign,

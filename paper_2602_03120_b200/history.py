@@ -31,7 +31,7 @@ class SeedHistory:
         return seeds, fitness, len(self._seeds)
 
     def push(self, seeds_now, fitness_now) -> None:
-        """Algorithm 2, "Enqueue(H, (S_t, F_t))": the oldest generation leaves once the window is full."""
+        """Algorithm 2, last line (the current seeds and rewards join the history): the oldest generation leaves once the window is full."""
         s_now, f_now = self._check(seeds_now, fitness_now)
         if self.window == 0:
             return

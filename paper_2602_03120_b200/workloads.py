@@ -10,7 +10,7 @@ and decoder-shaped weight sets (1.5B / 7B INT4, 7B INT8, 8B INT4) whose linear l
 take the geometry of the models the paper fine-tunes (Sec. 4.1, App. C); the paper's
 GPTQ checkpoints and task rewards are replaced by uniform random codes, lognormal
 scales and Gaussian / Student-t rewards that are z-scored per generation
-(Algorithm 1, "Normalize reward for population").
+(Algorithm 1, the reward-normalisation line of the population loop).
 """
 from __future__ import annotations
 
