@@ -380,7 +380,8 @@ def main():
     alu_peak = SM_COUNT * LANES_PER_SM * sm_mhz * 1e6
     achieved = upd_ops_per_launch / upd_s_per_launch
     bytes_per_launch = 2 * wl.packed_bytes(cfg.bits, model.numel) * args.steps / n_upd_launches
-    traffic = None if (DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE is None or quad or args.antithetic) else DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE * bytes_per_launch
+    # the capture was taken on the INT4 kernel in the default noise mode with independent members: other kernels get no figure
+    traffic = None if (DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE is None or quad or args.antithetic or cfg.bits != 4) else DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE * bytes_per_launch
     # scheduler cycles per (warp, sample): launch time x clock x schedulers / warp-samples of the launch
     warp_samples = model.numel * n_seeds * G * args.steps / n_upd_launches / 32.0
     cycles_per_warp_sample = upd_s_per_launch * sm_mhz * 1e6 * SM_COUNT * 4 / warp_samples

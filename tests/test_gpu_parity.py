@@ -710,3 +710,31 @@ def test_calls_run_on_the_callers_stream(qo, qes):
         assert not done.query(), "the call waited for the stream"
         s1.synchronize()
         assert torch.equal(w, want)
+
+
+def test_weight_unit_sigma_with_extreme_scales(qo, qes):
+    """sigma in weight units over scales at the ends of binary16: zero (sigma / 0 = +inf acts as 2^40: every
+    non-zero sample saturates the 4-bit range, a zero sample stays zero), the smallest subnormal, the largest finite
+    value, and an ordinary one -- perturbation bit for bit, update and history loop within the usual rules."""
+    import torch
+    rows, cols, N, K = 8, 256, 6, 2
+    for bits, group in ((4, 64), (8, 0)):
+        to, tg, packed, _ = _case(qo, qes, bits, rows, cols, group=group, off=32 * 11)
+        n_scales = rows * (cols // group) if group else rows
+        scales = np.resize(np.array([0.0, 2.0 ** -24, 65504.0, 0.0125], np.float16), n_scales)
+        for sigma in (0.02, 1e29):
+            kw = dict(sigma=sigma, lr=2.0 * sigma, gamma=0.9, n_pop=N, sigma_unit=1)
+            ho, hg = _hp(qo, qes, **kw)
+            seeds, fit = wl.draw_seeds(K + 1, N, stream=91), wl.draw_fitness(K + 1, N, stream=91)
+            wp = _dev(np.zeros_like(packed))
+            qes.qes_perturb(tg, _dev(packed), wp, _dev(scales), int(seeds[0, 0]), hg)
+            assert np.array_equal(_host(wp), qo.pack(bits, qo.perturb(to, packed, scales, int(seeds[0, 0]), ho)))
+            w = _dev(packed)
+            qes.qes_update(tg, w, _dev(scales), _dev(seeds), _dev(fit), K, None, hg)
+            ref = qo.update(to, packed, scales, seeds, fit, K, ho)
+            _compare_update(qo, _host(w), bits, ref, f"extreme scales, sigma {sigma}")
+            res = torch.empty(rows * cols, dtype=torch.float32, device="cuda")
+            qes.qes_replay_residual(tg, _dev(packed), _dev(scales), _dev(seeds[:K]), _dev(fit[:K]), K, hg, res)
+            rr = qo.replay_residual(to, packed, scales, seeds[:K], fit[:K], K, ho)
+            far = rr["band"] >= BAND
+            assert np.abs(_host(res).astype(np.float64) - rr["e"])[far].max(initial=0.0) <= TOL
