@@ -55,7 +55,8 @@ typedef enum {
     QES_ERR_BAD_HPARAM = -5,  /* sigma <= 0, n_pop <= 0 (or odd with antithetic pairs), K < 0 or K > QES_MAX_K, gamma outside [0,1], qmin >= qmax, range outside the code width */
     QES_ERR_BAD_MODE = -6,    /* unknown sigma_unit / boundary_mode / antithetic / residual_f16 / noise_mode, residual_inout given with K > 0, qes_perturb_pair without antithetic, or its two outputs the same buffer */
     QES_ERR_CUDA = -7,        /* the launch reported a CUDA error (cudaGetLastError) */
-    QES_ERR_TOO_LARGE = -8    /* more seeds per generation than the shared-memory staging holds (1066: members, or antithetic pairs) */
+    QES_ERR_TOO_LARGE = -8    /* a fixed capacity is exceeded: more seeds per generation than the shared-memory staging holds (1066: members,
+                                 or antithetic pairs), or more thread blocks than the static probe array has slots for */
 } qes_status;
 
 enum { QES_MAX_K = 1 << 20 };   /* largest replay depth K accepted */
@@ -239,6 +240,27 @@ int qes_gemv_perturbed(const qes_tensor_desc* desc, const void* w, const void* s
  *         20 lg2.approx.f32  21 sin.approx.f32  22 sqrt.approx.f32  23 cvt.rn.f32.s8
  */
 int qes_pipe_probe(int32_t kind, int32_t iters, void* sink_dev, float* ms_out, double* ops_out);
+
+/*
+ * The same probes for a caller that cannot allocate device memory (the paper has no counterpart for this either).
+ * qes_pipe_probe wants a device buffer from its caller and creates CUDA events; a process whose GPU memory is
+ * handed out entirely by some other allocator (an inference server that reserves the whole device at start-up, a
+ * plug-in that runs inside someone else's memory pool), or one that is forbidden to allocate once it is serving,
+ * has neither.  This entry point allocates nothing, on the device or through the CUDA runtime: the sink and one
+ * pair of time stamps per thread block live in a static device array of 8194 x 8 bytes (64 KiB) that is part of the
+ * library and stays on every GPU that has loaded it until the process ends.  Elapsed time is the last block's end
+ * minus the first block's start on the GPU's global nanosecond timer.
+ *   kind, iters   as for qes_pipe_probe.
+ *   ctas_per_sm   thread blocks per SM (qes_pipe_probe uses 8).  The grid is SMs x ctas_per_sm blocks and must not
+ *                 exceed the 4096 blocks the array has time slots for: QES_ERR_TOO_LARGE otherwise, nothing launched.
+ *   ms_out, ops_out   HOST pointers, as for qes_pipe_probe.
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that device
+ * current); make that first call before any stream capture begins.  Every call uses the same array and finds the
+ * previous call's time stamps in it; the slots it is going to read are cleared first.  Two calls that overlap on the
+ * same GPU (from two threads or processes sharing the context) would write the same slots and race: issue them one
+ * at a time.  Runs on the default stream and synchronises.
+ */
+int qes_pipe_probe_static(int32_t kind, int32_t iters, int32_t ctas_per_sm, float* ms_out, double* ops_out);
 
 const char* qes_strerror(int status);
 int qes_version(void);

@@ -124,6 +124,8 @@ def load() -> C.CDLL:
         lib.qes_gemv_perturbed.argtypes = [C.POINTER(_TensorDesc), vp, vp, u64, C.POINTER(_HParams), vp, vp, vp]
         lib.qes_pipe_probe.restype = C.c_int
         lib.qes_pipe_probe.argtypes = [i32, i32, vp, C.POINTER(C.c_float), C.POINTER(C.c_double)]
+        lib.qes_pipe_probe_static.restype = C.c_int
+        lib.qes_pipe_probe_static.argtypes = [i32, i32, i32, C.POINTER(C.c_float), C.POINTER(C.c_double)]
         lib.qes_strerror.restype = C.c_char_p
         lib.qes_strerror.argtypes = [C.c_int]
         lib.qes_version.restype = C.c_int
@@ -307,4 +309,12 @@ def qes_pipe_probe(kind: int, iters: int = 4096):
     ms, ops = C.c_float(0), C.c_double(0)
     torch.cuda.synchronize()
     _check(load().qes_pipe_probe(kind, iters, sink.data_ptr(), C.byref(ms), C.byref(ops)))
+    return ops.value / (ms.value * 1e-3), ms.value
+
+
+def qes_pipe_probe_static(kind: int, iters: int = 4096, ctas_per_sm: int = 8):
+    """qes_pipe_probe without any allocation: scratch and timing live in a static device array inside the library
+    (for callers whose device memory belongs to another allocator).  Returns (lane-operations per second, ms)."""
+    ms, ops = C.c_float(0), C.c_double(0)
+    _check(load().qes_pipe_probe_static(kind, iters, ctas_per_sm, C.byref(ms), C.byref(ops)))
     return ops.value / (ms.value * 1e-3), ms.value

@@ -794,7 +794,7 @@ const char* qes_strerror(int status) {
         case QES_ERR_BAD_HPARAM: return "hyper-parameter, replay depth or code range out of bounds";
         case QES_ERR_BAD_MODE: return "unknown mode, stored residual combined with K > 0, or a pair call without antithetic set";
         case QES_ERR_CUDA: return "CUDA reported an error at launch";
-        case QES_ERR_TOO_LARGE: return "n_pop exceeds the shared-memory staging limit";
+        case QES_ERR_TOO_LARGE: return "a fixed capacity is exceeded: seeds per generation above the shared-memory staging limit, or more thread blocks than the static probe array holds";
         default: return "unknown status";
     }
 }

@@ -2,6 +2,7 @@
 // Each probe runs kChains independent dependent-chains of one PTX instruction per thread on a
 // grid that fills every SM, and reports lane-operations and elapsed device time.
 #include <cstdint>
+#include <mutex>
 #include <cuda_runtime.h>
 #include "../../include/qes.h"
 
@@ -226,6 +227,175 @@ extern "C" int qes_pipe_probe(int32_t kind, int32_t iters, void* sink_dev, float
         case 21: return run_probe<21>(iters, sink, ms_out, ops_out);
         case 22: return run_probe<22>(iters, sink, ms_out, ops_out);
         case 23: return run_probe<23>(iters, sink, ms_out, ops_out);
+        default: return QES_ERR_BAD_MODE;
+    }
+}
+
+// ---- the same probes for callers that cannot allocate device memory ------------------------------------------
+// qes_pipe_probe needs a device buffer from its caller (the sink that keeps the chains live) and creates two CUDA
+// events.  A process whose device memory is wholly owned by another allocator, or one that must not allocate after
+// start-up, cannot supply either.  This variant keeps everything it needs in one static device array that is part
+// of the library image: word 0 is the sink, and each thread block records the global timer at its start and end in
+// its own pair of words, from which the host takes last end - first start.  The array lives on every GPU that loads
+// the library, until the process exits.
+namespace {
+
+constexpr int kStaticProbeMaxCtas = 4096;                       // thread blocks the time slots cover
+constexpr int kStaticProbeWords = 2 + 2 * kStaticProbeMaxCtas;  // 8194 x 8 B = 64.02 KiB per GPU
+static __device__ __align__(256) unsigned long long g_static_probe_scratch[kStaticProbeWords];
+
+constexpr int kStaticProbeMaxDevices = 64;
+std::mutex g_static_probe_mutex;
+unsigned long long* g_static_probe_address[kStaticProbeMaxDevices] = {};   // device address of the array, per device
+
+// In host code the array's name only stands for the symbol: the device address has to be asked for, once per
+// device and with that device current.
+int static_probe_scratch(unsigned long long** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return QES_ERR_CUDA; }
+    if (dev < 0 || dev >= kStaticProbeMaxDevices) return QES_ERR_TOO_LARGE;
+    std::lock_guard<std::mutex> lock(g_static_probe_mutex);
+    if (g_static_probe_address[dev] == nullptr) {
+        void* address = nullptr;
+        if (cudaGetSymbolAddress(&address, g_static_probe_scratch) != cudaSuccess || address == nullptr) {
+            cudaGetLastError();
+            return QES_ERR_CUDA;
+        }
+        g_static_probe_address[dev] = reinterpret_cast<unsigned long long*>(address);
+    }
+    *out = g_static_probe_address[dev];
+    return QES_OK;
+}
+
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// FORM 0: kChains chains of step<KIND>; 1: Philox rounds (kind 8); 2 / 3: wide multiply-add / wide multiply + xor3
+// (kinds 18 / 19) -- the arithmetic of the probes above, with the block's start and end times kept in `scratch`.
+template <int KIND, int FORM>
+__global__ void __launch_bounds__(kProbeThreads) static_probe_kernel(int iters, uint32_t a, uint32_t b, unsigned long long* scratch) {
+    const unsigned long long t0 = global_timer_ns();
+    uint32_t acc = 0;
+    if (FORM <= 1) {
+        uint32_t x[kChains];
+#pragma unroll
+        for (int c = 0; c < kChains; ++c) x[c] = threadIdx.x * 2654435761u + c * 40503u + blockIdx.x + 0x3f800001u;
+        if (FORM == 1) {
+            for (int it = 0; it < iters; ++it) {
+#pragma unroll
+                for (int c = 0; c < kChains; c += 4) {
+                    unsigned long long p0 = (unsigned long long)0xD2511F53u * x[c];
+                    unsigned long long p1 = (unsigned long long)0xCD9E8D57u * x[c + 2];
+                    uint32_t n0 = (uint32_t)(p1 >> 32) ^ x[c + 1] ^ a;
+                    uint32_t n2 = (uint32_t)(p0 >> 32) ^ x[c + 3] ^ b;
+                    x[c + 1] = (uint32_t)p1; x[c + 3] = (uint32_t)p0; x[c] = n0; x[c + 2] = n2;
+                }
+                a += 0x9E3779B9u; b += 0xBB67AE85u;
+            }
+        } else {
+            for (int it = 0; it < iters; ++it) {
+#pragma unroll
+                for (int c = 0; c < kChains; ++c) x[c] = step<KIND>(x[c], a, b);
+            }
+        }
+#pragma unroll
+        for (int c = 0; c < kChains; ++c) acc ^= x[c];
+    } else {
+        unsigned long long w[kChains];
+#pragma unroll
+        for (int c = 0; c < kChains; ++c)
+            w[c] = ((unsigned long long)(threadIdx.x * 2654435761u + c * 40503u) << 32) | (blockIdx.x + 0x3f800001u + c);
+        for (int it = 0; it < iters; ++it) {
+#pragma unroll
+            for (int c = 0; c < kChains; ++c) {
+                if (FORM == 2) {
+                    asm volatile("mad.wide.u32 %0, %1, %2, %0;" : "+l"(w[c]) : "r"((uint32_t)w[c]), "r"(a));
+                } else {
+                    unsigned long long p;
+                    asm volatile("mul.wide.u32 %0, %1, %2;" : "=l"(p) : "r"((uint32_t)w[c]), "r"(a));
+                    w[c] = (uint32_t)(p >> 32) ^ (uint32_t)p ^ b;
+                }
+            }
+        }
+#pragma unroll
+        for (int c = 0; c < kChains; ++c) acc ^= (uint32_t)w[c] ^ (uint32_t)(w[c] >> 32);
+    }
+    if (acc == 0x12345u) scratch[0] = acc;   // keeps the chains live; practically never taken
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        scratch[2 + 2 * blockIdx.x] = t0;
+        scratch[3 + 2 * blockIdx.x] = global_timer_ns();
+    }
+}
+
+template <int KIND, int FORM>
+int run_static_probe(int iters, int blocks, float* ms_out, double* ops_out) {
+    unsigned long long* scratch = nullptr;
+    int rc = static_probe_scratch(&scratch);
+    if (rc != QES_OK) return rc;
+    const size_t used = (size_t)(2 + 2 * blocks) * sizeof(unsigned long long);
+    static_probe_kernel<KIND, FORM><<<blocks, kProbeThreads>>>(iters / 8 + 1, 0x9E3779B9u, 0x3f7ffff0u, scratch);   // warm-up
+    // every call shares the array and finds the previous call's times in it: the slots start from zero, so that a
+    // block that did not run shows as a zero end time
+    if (cudaMemsetAsync(scratch, 0, used, 0) != cudaSuccess) { cudaGetLastError(); return QES_ERR_CUDA; }
+    static_probe_kernel<KIND, FORM><<<blocks, kProbeThreads>>>(iters, 0x9E3779B9u, 0x3f7ffff0u, scratch);
+    static thread_local unsigned long long host[kStaticProbeWords];
+    if (cudaMemcpy(host, scratch, used, cudaMemcpyDeviceToHost) != cudaSuccess || cudaGetLastError() != cudaSuccess) {
+        cudaGetLastError();
+        return QES_ERR_CUDA;
+    }
+    unsigned long long first = ~0ull, last = 0ull;
+    for (int b = 0; b < blocks; ++b) {
+        if (host[3 + 2 * b] == 0ull) return QES_ERR_CUDA;
+        if (host[2 + 2 * b] < first) first = host[2 + 2 * b];
+        if (host[3 + 2 * b] > last) last = host[3 + 2 * b];
+    }
+    *ms_out = (float)((double)(last - first) * 1e-6);
+    const double per_iter = (KIND == 8) ? (kChains / 4) * 4.0 : (double)kChains;
+    *ops_out = (double)blocks * kProbeThreads * (double)iters * per_iter;
+    return QES_OK;
+}
+
+}  // namespace
+
+extern "C" int qes_pipe_probe_static(int32_t kind, int32_t iters, int32_t ctas_per_sm, float* ms_out, double* ops_out) {
+    if (ms_out == nullptr || ops_out == nullptr) return QES_ERR_NULL_PTR;
+    if (iters <= 0 || iters > (1 << 24) || ctas_per_sm <= 0) return QES_ERR_BAD_HPARAM;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+        cudaGetLastError();
+        return QES_ERR_CUDA;
+    }
+    if ((int64_t)sms * ctas_per_sm > kStaticProbeMaxCtas) return QES_ERR_TOO_LARGE;   // more blocks than the array has time slots
+    const int blocks = sms * ctas_per_sm;
+    switch (kind) {
+        case 0: return run_static_probe<0, 0>(iters, blocks, ms_out, ops_out);
+        case 1: return run_static_probe<1, 0>(iters, blocks, ms_out, ops_out);
+        case 2: return run_static_probe<2, 0>(iters, blocks, ms_out, ops_out);
+        case 3: return run_static_probe<3, 0>(iters, blocks, ms_out, ops_out);
+        case 4: return run_static_probe<4, 0>(iters, blocks, ms_out, ops_out);
+        case 5: return run_static_probe<5, 0>(iters, blocks, ms_out, ops_out);
+        case 6: return run_static_probe<6, 0>(iters, blocks, ms_out, ops_out);
+        case 7: return run_static_probe<7, 0>(iters, blocks, ms_out, ops_out);
+        case 8: return run_static_probe<8, 1>(iters, blocks, ms_out, ops_out);
+        case 9: return run_static_probe<9, 0>(iters, blocks, ms_out, ops_out);
+        case 10: return run_static_probe<10, 0>(iters, blocks, ms_out, ops_out);
+        case 11: return run_static_probe<11, 0>(iters, blocks, ms_out, ops_out);
+        case 12: return run_static_probe<12, 0>(iters, blocks, ms_out, ops_out);
+        case 13: return run_static_probe<13, 0>(iters, blocks, ms_out, ops_out);
+        case 14: return run_static_probe<14, 0>(iters, blocks, ms_out, ops_out);
+        case 15: return run_static_probe<15, 0>(iters, blocks, ms_out, ops_out);
+        case 16: return run_static_probe<16, 0>(iters, blocks, ms_out, ops_out);
+        case 17: return run_static_probe<17, 0>(iters, blocks, ms_out, ops_out);
+        case 18: return run_static_probe<18, 2>(iters, blocks, ms_out, ops_out);
+        case 19: return run_static_probe<19, 3>(iters, blocks, ms_out, ops_out);
+        case 20: return run_static_probe<20, 0>(iters, blocks, ms_out, ops_out);
+        case 21: return run_static_probe<21, 0>(iters, blocks, ms_out, ops_out);
+        case 22: return run_static_probe<22, 0>(iters, blocks, ms_out, ops_out);
+        case 23: return run_static_probe<23, 0>(iters, blocks, ms_out, ops_out);
         default: return QES_ERR_BAD_MODE;
     }
 }

@@ -35,7 +35,7 @@ def test_every_declared_symbol_is_exported(lib):
     names = re.findall(r"^(?:int|const char\*)\s+(qes_\w+)\s*\(", header, flags=re.M)
     assert set(names) >= {"qes_perturb", "qes_update", "qes_replay_residual", "qes_perturb_pair", "qes_gaussian_factors", "qes_pipe_probe",
                           "qes_gaussian_estimates", "qes_estimate_bounds", "qes_pair_deltas", "qes_gemv", "qes_gemv_perturbed",
-                          "qes_replay_fidelity", "qes_strerror", "qes_version"}
+                          "qes_replay_fidelity", "qes_pipe_probe_static", "qes_strerror", "qes_version"}
     for n in names:
         assert hasattr(lib, n), n
     assert lib.qes_version() >= 100
