@@ -16,7 +16,7 @@
  * Conventions shared by all entry points
  *  - Pointers named w*, scales*, seeds, fitness, residual*, stats are DEVICE pointers owned by the
  *    caller; the two structs are HOST pointers read during the call.  The library allocates
- *    nothing, keeps no state between calls, enqueues its kernel on `cuda_stream` (a cudaStream_t
+ *    nothing, keeps no state between calls (qes_pipe_probe_static aside: it owns a static device array), enqueues its kernel on `cuda_stream` (a cudaStream_t
  *    passed as void*; NULL = the legacy default stream) and returns without synchronising.
  *  - Weights: row-major [rows, cols].  bits == 4: two codes per byte, even column in the low
  *    nibble, two's complement; bits == 8: one signed byte per code.  The base address must be
