@@ -738,3 +738,39 @@ def test_weight_unit_sigma_with_extreme_scales(qo, qes):
             rr = qo.replay_residual(to, packed, scales, seeds[:K], fit[:K], K, ho)
             far = rr["band"] >= BAND
             assert np.abs(_host(res).astype(np.float64) - rr["e"])[far].max(initial=0.0) <= TOL
+
+
+def test_tensor_with_more_than_2_pow_32_codes(qo, qes):
+    """One INT4 tensor of 2^32 + 2^20 codes (2 GiB packed): element and chunk indices pass 32 bits inside a single
+    launch.  Perturbation and a small stateless update, checked on sampled words that include the last ones."""
+    import torch
+    rows, cols = (1 << 17) + 32, 1 << 15
+    n = rows * cols
+    assert n > (1 << 32)
+    off = 32 * 5
+    g = torch.Generator(device="cuda"); g.manual_seed(5)
+    w0 = torch.randint(0, 256, (n // 2,), dtype=torch.uint8, device="cuda", generator=g)
+    idx = np.unique(np.concatenate([wl.sample_elements(n, 4096, stream=321),
+                                    (np.arange(64)[:, None] * 32 + np.arange(32)[None, :]).reshape(-1) + ((1 << 32) - 1024)]))
+    words = idx.reshape(-1, 32)[:, 0] // 32
+    assert idx[-1] == n - 1 and (idx > (1 << 32)).sum() > 1000
+    widx = torch.from_numpy(words).cuda()
+    before = w0.view(-1, 16)[widx].cpu().numpy()
+    sparse = np.zeros(n // 2, np.uint8)                       # untouched pages cost nothing
+    sparse.reshape(-1, 16)[words] = before
+    to = qo.Tensor(bits=4, rows=rows, cols=cols, elem_offset=off)
+    tg = qes.TensorDesc(bits=4, rows=rows, cols=cols, elem_offset=off)
+    N, K = 2, 1
+    ho, hg = _hp(qo, qes, sigma=0.5, lr=1.0, gamma=0.9, n_pop=N)
+    seeds, fit = wl.draw_seeds(K + 1, N, stream=322), wl.draw_fitness(K + 1, N, stream=322)
+    out = torch.empty_like(w0)
+    qes.qes_perturb(tg, w0, out, None, int(seeds[0, 0]), hg)
+    got_p = qo.unpack(4, out.view(-1, 16)[widx].cpu().numpy().reshape(-1), idx.size)
+    assert np.array_equal(got_p, qo.perturb(to, sparse, None, int(seeds[0, 0]), ho, idx=idx))
+    del out
+    qes.qes_update(tg, w0, None, _dev(seeds), _dev(fit), K, None, hg)
+    ref = qo.update(to, sparse, None, seeds, fit, K, ho, idx=idx)
+    got = qo.unpack(4, w0.view(-1, 16)[widx].cpu().numpy().reshape(-1), idx.size)
+    near = ref["band"] < BAND
+    assert not np.any((got != ref["w_new"]) & ~near)
+    assert (got != qo.unpack(4, before.reshape(-1), idx.size)).any()
